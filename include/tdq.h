@@ -1,0 +1,163 @@
+/*
+ * tdq.h -- C ABI of the COD-TDQ hot path on NVIDIA B200 (sm_100a).
+ *
+ * The library quantizes token activations with token-group scales (DSTG) whose clip
+ * radius is projected by two bounds (DCRP), quantizes weights per output channel, and
+ * runs the W4A4 linear layer on the 4-bit codes.
+ *
+ * Conventions shared by every call
+ *   - Unless a parameter is marked HOST, pointers are DEVICE pointers owned by the caller.
+ *     The library allocates nothing, frees nothing and keeps no pointer after the call.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL is the
+ *     default stream) and the call returns without waiting for it.
+ *   - Arguments are checked on the host before anything is launched.  A bad argument
+ *     returns an error code and launches nothing.  Nothing throws, aborts or traps.
+ *   - Kernels whose threads wait on each other give every wait an iteration limit.  A
+ *     wait that runs out writes a code into the call's workspace and the kernel returns;
+ *     tdq_workspace_status() reads that word back.
+ *   - Non-finite inputs (NaN, Inf) give unspecified codes; they never fault.
+ *
+ * Notation (the paper's): M = B*N tokens, C = I input channels, O output channels,
+ * g group size, K = C_pad / g groups per token with C_pad = g * ceil(C / g),
+ * q_max = 7, q_min = -8.
+ */
+#ifndef TDQ_H_
+#define TDQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    TDQ_OK = 0,
+    TDQ_ERR_INVALID_ARG = 1,    /* null pointer, non-positive size, parameter out of range   */
+    TDQ_ERR_UNSUPPORTED = 2,    /* a legal request this build has no kernel for              */
+    TDQ_ERR_ALIGNMENT = 3,      /* a pointer or stride misses the alignment stated below     */
+    TDQ_ERR_WORKSPACE = 4,      /* workspace missing or smaller than the size query returns  */
+    TDQ_ERR_CUDA = 5,           /* a CUDA runtime or driver call failed                      */
+    TDQ_ERR_DEVICE_TIMEOUT = 6  /* a bounded device-side wait ran out (see workspace status) */
+} tdq_status;
+
+typedef enum { TDQ_F32 = 0, TDQ_BF16 = 1 } tdq_dtype;
+
+/* Which DCRP bounds take part in the projection (Algorithm S1 step 4; the ablation
+ * variants of Table S6).  Both = COD-TDQ, neither = DSTG only. */
+#define TDQ_ENABLE_C1 1u  /* step-to-dispersion bound, Eq. 10 */
+#define TDQ_ENABLE_C2 2u  /* zero-bin mass bound, Eq. 11      */
+
+typedef struct {
+    int32_t group_size;      /* g, even, 2..4096; default 32.  g == C_pad gives one scale per token */
+    float tau;               /* C1: Delta_k / sigma_k <= tau, tau > 0; default 1.0                   */
+    float zr;                /* C2: zero-bin mass bound in (0,1]; default 0.2; rank ceil(zr*g)       */
+    float base_percentile;   /* p in (0,1]; 1.0 = max-abs base radius, else rank ceil(p*g) (Eq. 6)   */
+    uint32_t flags;          /* TDQ_ENABLE_C1 | TDQ_ENABLE_C2                                        */
+} tdq_act_params;
+
+/* The paper's shared setting (g, tau, zr) = (32, 1.0, 0.2), max-abs base radius, both bounds. */
+void tdq_default_act_params(tdq_act_params* p /* HOST, out */);
+
+/*
+ * Token-group dual-constraint activation quantizer: Algorithm S1 steps 1-7 (Eq. 5-12).
+ * For every token m and channel group k:
+ *   c_base = max |x| (or the ceil(p*g)-th smallest |x|);  sigma = population std + 1e-12;
+ *   thr = ceil(zr*g)-th smallest |x|;  c = max(min(c_base, 7*tau*sigma, 14*thr), 1e-8);
+ *   Delta = max(c/7, 1e-8);  q = clip(round_half_even(clip(x,-c,c) / Delta), -8, 7).
+ * Channels C..C_pad-1 are zeros; they take part in the statistics and get code 0.
+ *
+ *   x          [B*N rows, C] row-major, x_dtype, consecutive rows row_stride_elems apart
+ *              (>= C).  No alignment is required; 16-byte aligned x with C % 32 == 0,
+ *              row_stride_elems % 8 == 0 and g == 32 takes the fast kernel.
+ *   codes      [B*N, C_pad/2] bytes; byte j of a row holds channel 2j in its low nibble
+ *              and channel 2j+1 in its high nibble, two's complement.
+ *   scale      [B*N, K] float32, Delta_k.
+ *   offset     NULL, or [B*N, K] float32 that is filled with 0 (the grid is symmetric:
+ *              the paper's quantizer has no zero point).
+ * Errors: TDQ_ERR_INVALID_ARG for null x/p/codes/scale, B,N < 0, C <= 0, stride < C, odd or
+ * out-of-range g, tau <= 0, zr or p outside (0,1].  B*N == 0 is a no-op returning TDQ_OK.
+ */
+tdq_status tdq_quantize_act(const void* x, tdq_dtype x_dtype, int64_t B, int64_t N, int64_t C,
+                            int64_t row_stride_elems, const tdq_act_params* p /* HOST */,
+                            uint8_t* codes, float* scale, float* offset, void* cuda_stream);
+
+/*
+ * Static weight quantizer, Eq. 4 with absmax per-output-channel scales:
+ *   s_o = max(max_i |W[o,i]| / 7, 1e-8);  Q = clip(round_half_even(W / s_o), -8, 7).
+ *   w       [O, I] row-major, contiguous, w_dtype.
+ *   pad_to  the input dimension is zero-padded to I_pad, a multiple of pad_to (even;
+ *           pass the activation group size so both operands share C_pad).
+ *   wcodes  [O, I_pad/2] bytes, nibble order as for activations.   wscale [O] float32.
+ */
+tdq_status tdq_quantize_weight(const void* w, tdq_dtype w_dtype, int64_t O, int64_t I, int32_t pad_to,
+                               uint8_t* wcodes, float* wscale, void* cuda_stream);
+
+/*
+ * W4A4 linear layer, Algorithm S1 step 10 with x_hat = Delta_k q (Eq. 9) and
+ * W_hat = s_o Q_w (Eq. 4) substituted:
+ *   acc[m,o,k] = sum_{i in group k} q_x[m,i] * q_w[o,i]            (exact, int32)
+ *   y[m,o]     = s_o * sum_k Delta[m,k] * acc[m,o,k]  (+ bias[o])   (float32)
+ *   xcodes [M, I_pad/2], xscale [M, K], wcodes [O, I_pad/2], wscale [O], bias NULL or [O].
+ *   I_pad must be a multiple of group_size; group_size a multiple of 32 (the integer
+ *   tensor-core instruction contracts 32 codes at a time), at most 4096.
+ *   y      [M, O], y_dtype (float32 or bf16), rows y_row_stride elements apart (>= O).
+ *   acc_debug  NULL, or [M, O, K] int32 receiving every group's integer dot product
+ *              (for tests; slows the kernel down).
+ *   workspace  at least tdq_linear_workspace_bytes() bytes, 16-byte aligned.  Holds the
+ *              status word read by tdq_workspace_status().  The call clears it first, so
+ *              one workspace must not be shared by calls that overlap in time.
+ * Alignment: xcodes, wcodes 16 bytes; I_pad/2 % 16 == 0 is implied by g % 32 == 0.
+ */
+tdq_status tdq_w4a4_linear(const uint8_t* xcodes, const float* xscale, const uint8_t* wcodes,
+                           const float* wscale, const float* bias, int64_t M, int64_t I_pad, int64_t O,
+                           int32_t group_size, void* y, tdq_dtype y_dtype, int64_t y_row_stride,
+                           int32_t* acc_debug, void* workspace, size_t workspace_bytes,
+                           void* cuda_stream);
+
+/*
+ * Quantizer fused into the linear layer as the producer of its A operand: same result as
+ * tdq_quantize_act followed by tdq_w4a4_linear, but activation codes and scales never
+ * reach global memory.  Requires group_size == 32, C % 32 == 0 and the fast-path
+ * alignment of tdq_quantize_act; otherwise TDQ_ERR_UNSUPPORTED.
+ */
+tdq_status tdq_quant_linear_fused(const void* x, tdq_dtype x_dtype, int64_t B, int64_t N, int64_t C,
+                                  int64_t row_stride_elems, const tdq_act_params* p /* HOST */,
+                                  const uint8_t* wcodes, const float* wscale, const float* bias,
+                                  int64_t O, void* y, tdq_dtype y_dtype, int64_t y_row_stride,
+                                  void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * The two-kernel path with HOST input and output: copies x_host to x_dev, runs
+ * tdq_quantize_act and tdq_w4a4_linear, copies y_dev to y_host, all on cuda_stream.
+ * x_host / y_host should be page-locked for the copies to be asynchronous.  The device
+ * buffers are the caller's and sized as for the two calls (x_dev [B*N, C] dense).
+ */
+tdq_status tdq_quant_linear_host(const void* x_host /* HOST */, tdq_dtype x_dtype, int64_t B, int64_t N,
+                                 int64_t C, const tdq_act_params* p /* HOST */, const uint8_t* wcodes,
+                                 const float* wscale, const float* bias, int64_t O,
+                                 void* y_host /* HOST */, tdq_dtype y_dtype,
+                                 void* x_dev, uint8_t* codes_dev, float* scale_dev, void* y_dev,
+                                 void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Bytes of workspace tdq_w4a4_linear / tdq_quant_linear_fused need for this problem. */
+size_t tdq_linear_workspace_bytes(int64_t M, int64_t I_pad, int64_t O, int32_t group_size);
+
+/*
+ * Waits for cuda_stream, then reads the status word a linear call left in its workspace:
+ * TDQ_OK, or TDQ_ERR_DEVICE_TIMEOUT when a bounded wait inside the kernel ran out (the
+ * output of that call is then incomplete).  detail (HOST, nullable) receives the raw word:
+ * bits 0-7 name the wait that gave up, bits 8-31 the tile index.
+ */
+tdq_status tdq_workspace_status(const void* workspace, void* cuda_stream, uint32_t* detail /* HOST */);
+
+/* Static description of a status code. */
+const char* tdq_status_string(tdq_status s);
+
+/* Number of kernels this library has launched in the calling process (for accounting). */
+uint64_t tdq_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TDQ_H_ */

@@ -1,0 +1,201 @@
+"""ctypes binding of libtdq.so.  Argument marshalling only: every step runs in the library's
+CUDA kernels.  torch is used to allocate device memory and to name the current stream."""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtdq.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        "libtdq.so is missing: build it with `python -m paper_2604_16855_b200.build` "
+        "(there is no fallback implementation)")
+_lib = ctypes.CDLL(LIB_PATH)
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_DEVICE_TIMEOUT = range(7)
+F32, BF16 = 0, 1
+ENABLE_C1, ENABLE_C2 = 1, 2
+
+# every symbol include/tdq.h declares
+EXPORTS = ["tdq_default_act_params", "tdq_quantize_act", "tdq_quantize_weight", "tdq_w4a4_linear",
+           "tdq_quant_linear_fused", "tdq_quant_linear_host", "tdq_linear_workspace_bytes",
+           "tdq_workspace_status", "tdq_status_string", "tdq_kernel_launch_count"]
+
+
+class ActParams(ctypes.Structure):
+    _fields_ = [("group_size", ctypes.c_int32), ("tau", ctypes.c_float), ("zr", ctypes.c_float),
+                ("base_percentile", ctypes.c_float), ("flags", ctypes.c_uint32)]
+
+
+_i64, _i32, _vp, _sz = ctypes.c_int64, ctypes.c_int32, ctypes.c_void_p, ctypes.c_size_t
+_pp = ctypes.POINTER(ActParams)
+_lib.tdq_default_act_params.argtypes = [_pp]
+_lib.tdq_default_act_params.restype = None
+_lib.tdq_quantize_act.argtypes = [_vp, ctypes.c_int, _i64, _i64, _i64, _i64, _pp, _vp, _vp, _vp, _vp]
+_lib.tdq_quantize_act.restype = ctypes.c_int
+_lib.tdq_quantize_weight.argtypes = [_vp, ctypes.c_int, _i64, _i64, _i32, _vp, _vp, _vp]
+_lib.tdq_quantize_weight.restype = ctypes.c_int
+_lib.tdq_w4a4_linear.argtypes = [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp, ctypes.c_int, _i64,
+                                 _vp, _vp, _sz, _vp]
+_lib.tdq_w4a4_linear.restype = ctypes.c_int
+_lib.tdq_quant_linear_fused.argtypes = [_vp, ctypes.c_int, _i64, _i64, _i64, _i64, _pp, _vp, _vp, _vp, _i64,
+                                        _vp, ctypes.c_int, _i64, _vp, _sz, _vp]
+_lib.tdq_quant_linear_fused.restype = ctypes.c_int
+_lib.tdq_quant_linear_host.argtypes = [_vp, ctypes.c_int, _i64, _i64, _i64, _pp, _vp, _vp, _vp, _i64, _vp,
+                                       ctypes.c_int, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+_lib.tdq_quant_linear_host.restype = ctypes.c_int
+_lib.tdq_linear_workspace_bytes.argtypes = [_i64, _i64, _i64, _i32]
+_lib.tdq_linear_workspace_bytes.restype = _sz
+_lib.tdq_workspace_status.argtypes = [_vp, _vp, ctypes.POINTER(ctypes.c_uint32)]
+_lib.tdq_workspace_status.restype = ctypes.c_int
+_lib.tdq_status_string.argtypes = [ctypes.c_int]
+_lib.tdq_status_string.restype = ctypes.c_char_p
+_lib.tdq_kernel_launch_count.argtypes = []
+_lib.tdq_kernel_launch_count.restype = ctypes.c_uint64
+
+
+class TdqError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        super().__init__("%s: %s (status %d)" % (where, status_string(code), code))
+
+
+def lib():
+    """The loaded ctypes library (for callers that want the raw C ABI)."""
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return _lib.tdq_status_string(int(code)).decode()
+
+
+def kernel_launch_count() -> int:
+    return int(_lib.tdq_kernel_launch_count())
+
+
+def default_act_params() -> ActParams:
+    p = ActParams()
+    _lib.tdq_default_act_params(ctypes.byref(p))
+    return p
+
+
+def act_params(g=32, tau=1.0, zr=0.2, p=1.0, flags=ENABLE_C1 | ENABLE_C2) -> ActParams:
+    return ActParams(int(g), float(tau), float(zr), float(p), int(flags))
+
+
+def _check(code, where):
+    if code != OK:
+        raise TdqError(code, where)
+
+
+def _dtype_id(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError("tdq takes float32 or bfloat16 tensors, got %s" % t.dtype)
+
+
+def _stream(t: torch.Tensor):
+    return ctypes.c_void_p(torch.cuda.current_stream(t.device).cuda_stream)
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _need_cuda(*ts):
+    for t in ts:
+        if t is not None and not t.is_cuda:
+            raise ValueError("tdq runs on CUDA tensors only; there is no CPU path")
+
+
+def quantize_act(x: torch.Tensor, params: ActParams | None = None, *, codes=None, scale=None, offset=None):
+    """tdq_quantize_act on x [..., C] (last dim contiguous, rows equally spaced).
+
+    Returns (codes uint8 [M, C_pad/2], scale float32 [M, K])."""
+    _need_cuda(x)
+    p = params or default_act_params()
+    C = x.shape[-1]
+    x2 = x.reshape(-1, C)
+    if x2.stride(-1) != 1:
+        raise ValueError("the channel axis must be contiguous")
+    M = x2.shape[0]
+    g = p.group_size
+    K = (C + g - 1) // g
+    if codes is None:
+        codes = torch.empty((M, K * g // 2), dtype=torch.uint8, device=x.device)
+    if scale is None:
+        scale = torch.empty((M, K), dtype=torch.float32, device=x.device)
+    stride = x2.stride(0) if M > 1 else C
+    _check(_lib.tdq_quantize_act(_ptr(x2), _dtype_id(x2), 1, M, C, stride, ctypes.byref(p), _ptr(codes),
+                                 _ptr(scale), _ptr(offset), _stream(x)), "tdq_quantize_act")
+    return codes, scale
+
+
+def quantize_weight(w: torch.Tensor, pad_to: int = 32, *, wcodes=None, wscale=None):
+    """tdq_quantize_weight on w [O, I] (contiguous).  Returns (wcodes uint8 [O, I_pad/2], wscale [O])."""
+    _need_cuda(w)
+    w = w.contiguous()
+    O, I = w.shape
+    I_pad = (I + pad_to - 1) // pad_to * pad_to
+    if wcodes is None:
+        wcodes = torch.empty((O, I_pad // 2), dtype=torch.uint8, device=w.device)
+    if wscale is None:
+        wscale = torch.empty((O,), dtype=torch.float32, device=w.device)
+    _check(_lib.tdq_quantize_weight(_ptr(w), _dtype_id(w), O, I, pad_to, _ptr(wcodes), _ptr(wscale), _stream(w)),
+           "tdq_quantize_weight")
+    return wcodes, wscale
+
+
+def linear_workspace(M, I_pad, O, g, device) -> torch.Tensor:
+    n = int(_lib.tdq_linear_workspace_bytes(M, I_pad, O, g))
+    return torch.zeros((n,), dtype=torch.uint8, device=device)
+
+
+def w4a4_linear(xcodes, xscale, wcodes, wscale, bias=None, *, g=32, out_dtype=torch.float32, y=None,
+                acc_debug=None, workspace=None):
+    """tdq_w4a4_linear.  Returns y [M, O]."""
+    _need_cuda(xcodes, xscale, wcodes, wscale, bias)
+    M, half = xcodes.shape
+    I_pad = half * 2
+    O = wcodes.shape[0]
+    if y is None:
+        y = torch.empty((M, O), dtype=out_dtype, device=xcodes.device)
+    if workspace is None:
+        workspace = linear_workspace(M, I_pad, O, g, xcodes.device)
+    _check(_lib.tdq_w4a4_linear(_ptr(xcodes), _ptr(xscale), _ptr(wcodes), _ptr(wscale), _ptr(bias), M, I_pad, O, g,
+                                _ptr(y), _dtype_id(y), y.stride(0) if M > 0 else O, _ptr(acc_debug),
+                                _ptr(workspace), workspace.numel(), _stream(xcodes)), "tdq_w4a4_linear")
+    return y
+
+
+def quant_linear_fused(x, wcodes, wscale, bias=None, params: ActParams | None = None, *,
+                       out_dtype=torch.float32, y=None, workspace=None):
+    """tdq_quant_linear_fused: quantizer as the linear layer's A-operand producer.  Returns y [M, O]."""
+    _need_cuda(x, wcodes, wscale, bias)
+    p = params or default_act_params()
+    C = x.shape[-1]
+    x2 = x.reshape(-1, C)
+    M = x2.shape[0]
+    O = wcodes.shape[0]
+    if y is None:
+        y = torch.empty((M, O), dtype=out_dtype, device=x.device)
+    if workspace is None:
+        workspace = linear_workspace(M, wcodes.shape[1] * 2, O, p.group_size, x.device)
+    stride = x2.stride(0) if M > 1 else C
+    _check(_lib.tdq_quant_linear_fused(_ptr(x2), _dtype_id(x2), 1, M, C, stride, ctypes.byref(p), _ptr(wcodes),
+                                       _ptr(wscale), _ptr(bias), O, _ptr(y), _dtype_id(y), y.stride(0),
+                                       _ptr(workspace), workspace.numel(), _stream(x)), "tdq_quant_linear_fused")
+    return y
+
+
+def workspace_status(workspace: torch.Tensor):
+    """(status, detail word) left by the last linear call that used this workspace; synchronises."""
+    detail = ctypes.c_uint32(0)
+    st = _lib.tdq_workspace_status(_ptr(workspace), _stream(workspace), ctypes.byref(detail))
+    return int(st), int(detail.value)

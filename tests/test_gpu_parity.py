@@ -1,0 +1,220 @@
+"""GPU parity: every C-ABI entry point against the CPU oracle on the same seeded inputs.
+All tests call through the ctypes binding of libtdq.so; the rules are in parity_utils."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth_inputs as si
+from parity_utils import case_tensors, compare_quantizer, compare_y, to_cuda, unpack_codes
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def tdq():
+    from paper_2604_16855_b200 import tdq
+    return tdq
+
+
+def _quant_both(tdq, x_np, bf16, **kw):
+    """(oracle dict, gpu codes, gpu scale) for x_np [M, C] (float32, or uint16 bf16 bits)."""
+    g = kw.get("g", 32)
+    ref = oracle.quantize_act(x_np, **kw)
+    params = tdq.act_params(g=g, tau=kw.get("tau", 1.0), zr=kw.get("zr", 0.2), p=kw.get("p", 1.0),
+                            flags=kw.get("flags", 3))
+    codes, scale = tdq.quantize_act(to_cuda(x_np, bf16=bf16), params)
+    torch.cuda.synchronize()
+    return ref, codes.cpu().numpy(), scale.cpu().numpy()
+
+
+def _f32(x_np, bf16):
+    return si.bf16_bits_to_f32(x_np) if bf16 else x_np
+
+
+# ---------------------------------------------------------------------------------------
+# quantizer
+
+@pytest.mark.parametrize("idx", [1, 2, 3, 4])
+def test_quantizer_matches_oracle_on_workloads(tdq, idx):
+    case = si.config(idx)
+    x = case.x.reshape(-1, case.C)
+    ref, codes, scale = _quant_both(tdq, x, case.x_is_bf16)
+    rep = compare_quantizer(_f32(x, case.x_is_bf16), 32, ref, codes, scale)
+    print("cfg%d quantizer parity: %s" % (idx, rep))
+    assert rep["scale_exact_frac"] == 1.0
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("tau,zr,flags", [(1.0, 0.2, 3), (0.5, 0.2, 3), (0.25, 0.1, 3), (1.0, 0.5, 3),
+                                          (1.0, 0.2, 1), (1.0, 0.2, 2), (1.0, 0.2, 0), (0.3, 0.4, 3), (2.0, 1.0, 3)])
+def test_quantizer_fast_path_settings_and_c1_binding(tdq, bf16, tau, zr, flags):
+    xs = [si.dc_offset_tokens(M=700, C=96), si.config1().x.reshape(-1, 64), si.edge_rows(C=64)]
+    for x in xs:
+        if bf16:
+            x = si.f32_to_bf16_bits(x)
+        ref, codes, scale = _quant_both(tdq, x, bf16, tau=tau, zr=zr, flags=flags)
+        rep = compare_quantizer(_f32(x, bf16), 32, ref, codes, scale)
+        assert rep["scale_exact_frac"] == 1.0, rep
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("C,g", [(48, 32), (72, 32), (100, 32), (64, 16), (128, 64), (96, 96), (320, 320),
+                                 (70, 14), (4096, 4096), (30, 32)])
+def test_quantizer_generic_path_padding_and_group_sizes(tdq, bf16, C, g):
+    rng = np.random.default_rng(C * 1000 + g)
+    x = si.token_mixture(rng, 1, 37, C, sigma_log_std=0.5, bg_frac=0.1, bg_nu=3.0, bg_amp=20.0).reshape(-1, C)
+    x[::5] += 2.0                                    # some C1-bound groups
+    if bf16:
+        x = si.f32_to_bf16_bits(x)
+    for kw in (dict(), dict(p=0.9), dict(tau=0.5, zr=0.3)):
+        ref, codes, scale = _quant_both(tdq, x, bf16, g=g, **kw)
+        rep = compare_quantizer(_f32(x, bf16), g, ref, codes, scale)
+        assert rep["scale_max_rel"] <= 1e-6
+
+
+def test_quantizer_percentile_and_odd_rank_take_generic_kernel(tdq):
+    x = si.config1().x.reshape(-1, 64)
+    for kw in (dict(p=0.9), dict(zr=0.27), dict(zr=0.95, p=0.5)):
+        ref, codes, scale = _quant_both(tdq, x, False, **kw)
+        compare_quantizer(x, 32, ref, codes, scale)
+
+
+def test_quantizer_row_stride_offset_output_and_empty(tdq):
+    case = si.config2()
+    bits = case.x.reshape(-1, 64)[:1000]
+    wide = np.full((1000, 96), 0x7F7F, np.uint16)
+    wide[:, :64] = bits
+    xt = to_cuda(wide, bf16=True)[:, :64]            # row stride 96 elements, fast path
+    ref = oracle.quantize_act(bits)
+    off = torch.full((1000, 2), 5.0, device="cuda")
+    codes, scale = tdq.quantize_act(xt, offset=off)
+    compare_quantizer(si.bf16_bits_to_f32(bits), 32, ref, codes.cpu().numpy(), scale.cpu().numpy())
+    assert (off == 0).all()
+    wide2 = np.full((1000, 75), 0x7F7F, np.uint16)   # stride 75: unaligned rows -> generic kernel
+    wide2[:, :64] = bits
+    codes, scale = tdq.quantize_act(to_cuda(wide2, bf16=True)[:, :64])
+    compare_quantizer(si.bf16_bits_to_f32(bits), 32, ref, codes.cpu().numpy(), scale.cpu().numpy())
+    c0, s0 = tdq.quantize_act(torch.empty((0, 64), device="cuda"))
+    assert c0.shape == (0, 32) and s0.shape == (0, 2)
+
+
+def test_quantizer_does_not_write_outside_its_outputs(tdq):
+    x = to_cuda(si.config1().x.reshape(-1, 64)[:77])
+    codes = torch.full((77 * 32 + 64,), 0xAB, dtype=torch.uint8, device="cuda")
+    scale = torch.full((77 * 2 + 16,), -1.0, device="cuda")
+    tdq.quantize_act(x, codes=codes[32:32 + 77 * 32].view(77, 32), scale=scale[8:8 + 154].view(77, 2))
+    torch.cuda.synchronize()
+    assert (codes[:32] == 0xAB).all() and (codes[-32:] == 0xAB).all()
+    assert (scale[:8] == -1).all() and (scale[-8:] == -1).all()
+
+
+# ---------------------------------------------------------------------------------------
+# weight quantizer
+
+@pytest.mark.parametrize("O,I,bf16", [(64, 64, False), (256, 64, False), (40, 100, False), (960, 320, True), (3, 7, False)])
+def test_weight_quantizer_matches_oracle(tdq, O, I, bf16):
+    rng = np.random.default_rng(O + I)
+    w = si.weights(rng, O, I)
+    w[0] = 0.0
+    w_np = si.f32_to_bf16_bits(w) if bf16 else w
+    ref = oracle.quantize_weight(w_np, pad_to=32)
+    wc, ws = tdq.quantize_weight(to_cuda(w_np, bf16=bf16), 32)
+    np.testing.assert_array_equal(ws.cpu().numpy(), ref["scale"])
+    np.testing.assert_array_equal(wc.cpu().numpy(), ref["codes"])
+
+
+# ---------------------------------------------------------------------------------------
+# linear layer
+
+def _linear_case(tdq, x_np, bf16, w_np, g=32, bias=None, out_dtype=torch.float32, want_acc=True, rows=None, **kw):
+    xa = oracle.quantize_act(x_np, g=g, **kw)
+    wq = oracle.quantize_weight(w_np, pad_to=g)
+    xc, xs = to_cuda(xa["codes"]), to_cuda(xa["scale"])
+    wc, ws = to_cuda(wq["codes"]), to_cuda(wq["scale"])
+    M, O, K = xa["codes"].shape[0], w_np.shape[0], xa["scale"].shape[1]
+    acc = torch.full((M, O, K), 12345, dtype=torch.int32, device="cuda") if want_acc else None
+    b = None if bias is None else to_cuda(bias)
+    wsp = tdq.linear_workspace(M, K * g, O, g, "cuda")
+    y = tdq.w4a4_linear(xc, xs, wc, ws, b, g=g, out_dtype=out_dtype, acc_debug=acc, workspace=wsp)
+    st, detail = tdq.workspace_status(wsp)
+    assert st == tdq.OK, "device wait ran out: 0x%x" % detail
+    sel = slice(None) if rows is None else rows
+    ref = oracle.w4a4_linear(xa["codes"][sel], xa["scale"][sel], wq["codes"], wq["scale"], bias=bias, g=g,
+                             want_acc=want_acc)
+    if want_acc:
+        np.testing.assert_array_equal(acc.cpu().numpy()[sel], ref["acc"])     # bit-exact integer sums
+    return y.float().cpu().numpy()[sel], ref
+
+
+@pytest.mark.parametrize("idx", [1, 2])
+def test_linear_matches_oracle_small_workloads(tdq, idx):
+    case = si.config(idx)
+    x = case.x.reshape(-1, case.C)
+    if idx == 2:
+        x = x[:3000]
+    y, ref = _linear_case(tdq, x, case.x_is_bf16, case.w)
+    worst = compare_y(y, ref["y_d"])
+    print("cfg%d linear: worst err/tol %.3f" % (idx, worst))
+
+
+@pytest.mark.parametrize("M,C,O,g", [(1, 32, 8, 32), (129, 64, 65, 32), (300, 96, 200, 32), (257, 320, 130, 32),
+                                     (100, 128, 64, 64), (130, 256, 96, 128), (64, 768, 72, 768), (50, 100, 30, 32)])
+def test_linear_shapes_tails_bias_and_wide_groups(tdq, M, C, O, g):
+    rng = np.random.default_rng(M + C + O)
+    x = si.token_mixture(rng, 1, M, C, sigma_log_std=0.5, bg_frac=0.1, bg_nu=3.0, bg_amp=20.0).reshape(-1, C)
+    w = si.weights(rng, O, C)
+    bias = rng.standard_normal(O).astype(np.float32)
+    y, ref = _linear_case(tdq, x, False, w, g=g, bias=bias)
+    compare_y(y, ref["y_d"])
+
+
+def test_linear_bf16_output_and_row_stride(tdq):
+    case = si.config1()
+    x = case.x.reshape(-1, 64)
+    y, ref = _linear_case(tdq, x, False, case.w, out_dtype=torch.bfloat16, want_acc=False)
+    err = np.abs(y - ref["y_d"])
+    rms = np.sqrt((ref["y_d"] ** 2).mean(-1, keepdims=True))
+    assert (err <= 2.0 ** -8 * np.maximum(np.abs(ref["y_d"]), 1e-3 * rms) * 1.01).all()   # one bf16 rounding
+    xa = oracle.quantize_act(x)
+    wq = oracle.quantize_weight(case.w)
+    ybig = torch.full((256, 80), 7.0, device="cuda")
+    tdq.w4a4_linear(to_cuda(xa["codes"]), to_cuda(xa["scale"]), to_cuda(wq["codes"]), to_cuda(wq["scale"]),
+                    y=ybig[:, :64])
+    torch.cuda.synchronize()
+    compare_y(ybig[:, :64].cpu().numpy(), ref["y_d"])
+    assert (ybig[:, 64:] == 7.0).all()
+
+
+@pytest.mark.parametrize("idx", [3, 4])
+def test_linear_full_size_workloads_on_sampled_rows(tdq, idx):
+    case = si.config(idx)
+    x = case.x.reshape(-1, case.C)
+    rng = np.random.default_rng(idx)
+    rows = np.sort(np.concatenate([rng.choice(x.shape[0], 160, replace=False), [0, 127, 128, x.shape[0] - 1]]))
+    rows = np.unique(rows)
+    y, ref = _linear_case(tdq, x, case.x_is_bf16, case.w, want_acc=False, rows=rows)
+    worst = compare_y(y, ref["y_d"])
+    print("cfg%d linear (sampled %d rows): worst err/tol %.3f" % (idx, len(rows), worst))
+
+
+def test_quantize_then_linear_end_to_end_matches_oracle(tdq):
+    case = si.config3()
+    x = case.x.reshape(-1, case.C)[:1500]
+    xt = to_cuda(x, bf16=True)
+    wc, ws = tdq.quantize_weight(to_cuda(case.w))
+    codes, scale = tdq.quantize_act(xt)
+    y = tdq.w4a4_linear(codes, scale, wc, ws)
+    xa = oracle.quantize_act(x)
+    wq = oracle.quantize_weight(case.w)
+    ref = oracle.w4a4_linear(xa["codes"], xa["scale"], wq["codes"], wq["scale"])
+    np.testing.assert_array_equal(codes.cpu().numpy(), xa["codes"])
+    compare_y(y.cpu().numpy(), ref["y_d"])
+
+
+def test_sweep_layers_spot_check(tdq):
+    for li in (3, 11, 19, 31):                   # fc2 of each stage: the widest contraction of the stage
+        case = si.config5_layer(li, batch=1)
+        x = case.x.reshape(-1, case.C)[:512]
+        y, ref = _linear_case(tdq, x, True, case.w, want_acc=False)
+        compare_y(y, ref["y_d"])
