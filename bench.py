@@ -1,0 +1,343 @@
+"""Benchmark of the COD-TDQ hot path on B200: token-group quantizer -> W4A4 linear.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl tdq|reference] [--workload cfg4|cfg3|cfg2]
+
+A step is one pass of the whole path over one batch of the workload: tdq_quantize_act on X,
+then tdq_w4a4_linear on the codes (weights are quantized once, before timing: they are
+static).  The default workload is the ViT-B-style MLP fc1 case, X bf16 [32, 577, 768] and
+W [3072, 768], the largest of the single-layer workloads.  One JSON line is printed.
+
+  value / unit       quantizer throughput in GB/s: algorithmic bytes (2 B read + 0.5 B codes +
+                     0.125 B scale per element) / device time of the quantizer kernel, summed
+                     over all ranks.  The linear layer's TOPS and both roofline fractions are
+                     in "kernels"; ms_per_step is the whole step.
+  e2e                the same quantity through tdq_quant_linear_host with pinned HOST input and
+                     output, copies inside the timed region.
+  roofline           for the kernel that takes most of the step.
+  cpu_baseline       the CPU oracle on the host cores, on a bounded sample, rank 0, N=1 only.
+
+--impl reference times the CPU oracle as it stands (rank 0 only).
+Multi-GPU: rows are independent, every rank runs its own full batch (weak scaling, no
+collective on the data path); the time is the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import synth_inputs as si  # noqa: E402
+
+METRIC = "quantizer GB/s and W4A4 linear TOPS at 1 B200, % of HBM / INT8 roofline"
+L2_BYTES = 126 * 2 ** 20
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def workload(name):
+    return {"cfg2": si.config2, "cfg3": si.config3, "cfg4": si.config4}[name]()
+
+
+def quant_bytes(M, C, esize, g=32):
+    return M * C * esize + M * C // 2 + M * (C // g) * 4
+
+
+def linear_bytes(M, I, O, g=32, ysize=4):
+    return M * I // 2 + M * (I // g) * 4 + O * I // 2 + O * 4 + M * O * ysize
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, pw, reasons = [], [], [], set()
+        for l in self.lines:
+            f = [v.strip() for v in l.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); pw.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["no samples"])
+        # the busiest samples are the ones taken under load
+        load = sorted(sm)[len(sm) // 2:]
+        return dict(sm_mhz=float(np.median(load)), sm_max_mhz=float(max(mx)), power_w_max=float(max(pw)),
+                    samples=len(sm), reasons=sorted(reasons))
+
+
+def cpu_oracle_leg(case, rows, repeats=1):
+    """Times the oracle (quantizer + linear) on the first `rows` token rows.  Returns a dict."""
+    import oracle
+    x = case.x.reshape(-1, case.C)[:rows]
+    wq = oracle.quantize_weight(case.w, pad_to=32)
+    best_q, best_l = 1e30, 1e30
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        xa = oracle.quantize_act(x)
+        t1 = time.perf_counter()
+        oracle.w4a4_linear(xa["codes"], xa["scale"], wq["codes"], wq["scale"])
+        t2 = time.perf_counter()
+        best_q, best_l = min(best_q, t1 - t0), min(best_l, t2 - t1)
+    esize = 2 if case.x_is_bf16 else 4
+    return dict(rows=int(x.shape[0]), quant_s=best_q, linear_s=best_l,
+                quant_gbs=quant_bytes(x.shape[0], case.C, esize) / best_q / 1e9,
+                linear_tops=2.0 * x.shape[0] * case.C * case.O / best_l / 1e12,
+                cores=oracle.num_threads())
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    case = workload(args.workload)
+    rows = 2048
+    for _ in range(args.warmup):
+        cpu_oracle_leg(case, rows)
+    t0 = time.perf_counter()
+    legs = [cpu_oracle_leg(case, rows) for _ in range(args.steps)]
+    wall = time.perf_counter() - t0
+    qs = sum(l["quant_s"] for l in legs)
+    ls = sum(l["linear_s"] for l in legs)
+    esize = 2 if case.x_is_bf16 else 4
+    value = args.steps * quant_bytes(rows, case.C, esize) / qs / 1e9
+    sample = "first %d of %d token rows of %s per step, quantizer + linear" % (rows, case.M, case.name)
+    out = dict(metric=METRIC, impl="reference", value=value, unit="GB/s", n_gpus=args.gpus, steps=args.steps,
+               warmup=args.warmup, ms_per_step=1e3 * wall / args.steps, higher_is_better=True, scaling="weak",
+               vs_baseline=None, dtype="f32 quantizer / int32 contraction / f64 scaling", data="synthetic",
+               config=dict(workload=case.name, x=[int(v) for v in case.x.shape], w=[int(v) for v in case.w.shape],
+                           g=32, tau=1.0, zr=0.2, sample=sample),
+               kernels=dict(linear=dict(tops=2.0 * args.steps * rows * case.C * case.O / ls / 1e12)),
+               cpu_baseline=dict(value=value, unit="GB/s", cores=legs[0]["cores"], kind="oracle", sample=sample),
+               e2e=dict(value=value, unit="GB/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
+    print(json.dumps(out))
+
+
+def run_tdq(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2604_16855_b200 import tdq
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    case = workload(args.workload)
+    M, C, O = case.M, case.C, case.O
+    esize = 2 if case.x_is_bf16 else 4
+    x_host = torch.from_numpy(case.x.reshape(M, C).view(np.int16).copy()).view(torch.bfloat16) if case.x_is_bf16 \
+        else torch.from_numpy(case.x.reshape(M, C).copy())
+    w = torch.from_numpy(case.w).to(dev)
+    wcodes, wscale = tdq.quantize_weight(w, 32)
+
+    # rotating buffer sets: a step touches X, codes, scales and Y; keep the rotation larger than L2
+    step_bytes = quant_bytes(M, C, esize) + M * O * 4
+    nsets = max(2, int(np.ceil(2.5 * L2_BYTES / step_bytes)))
+    xs = [x_host.to(dev) for _ in range(nsets)]
+    codes = [torch.empty((M, C // 2), dtype=torch.uint8, device=dev) for _ in range(nsets)]
+    scales = [torch.empty((M, C // 32), dtype=torch.float32, device=dev) for _ in range(nsets)]
+    ys = [torch.empty((M, O), dtype=torch.float32, device=dev) for _ in range(nsets)]
+    wsp = tdq.linear_workspace(M, C, O, 32, dev)
+    params = tdq.default_act_params()
+
+    def step(i, ev=None):
+        s = i % nsets
+        if ev:
+            ev[0].record()
+        tdq.quantize_act(xs[s], params, codes=codes[s], scale=scales[s])
+        if ev:
+            ev[1].record()
+        tdq.w4a4_linear(codes[s], scales[s], wcodes, wscale, y=ys[s], workspace=wsp)
+        if ev:
+            ev[2].record()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    st, detail = tdq.workspace_status(wsp)
+    if st != tdq.OK:
+        raise RuntimeError("linear kernel reported a device-side timeout: 0x%x" % detail)
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    launches0 = tdq.kernel_launch_count()
+    barrier()
+    t_begin = torch.cuda.Event(enable_timing=True)
+    t_end = torch.cuda.Event(enable_timing=True)
+    t_begin.record()
+    for i in range(args.steps):
+        step(args.warmup + i, evs[i])
+    t_end.record()
+    barrier()
+    launches = tdq.kernel_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = t_begin.elapsed_time(t_end)
+    q_ms = sum(e[0].elapsed_time(e[1]) for e in evs)
+    l_ms = sum(e[1].elapsed_time(e[2]) for e in evs)
+
+    # end to end: pinned host X in, host Y out, through the host-buffer entry point
+    xh = x_host.pin_memory()
+    yh = torch.empty((M, O), dtype=torch.float32).pin_memory()
+    stream = torch.cuda.current_stream().cuda_stream
+    import ctypes
+
+    def e2e_step():
+        rc = tdq.lib().tdq_quant_linear_host(
+            ctypes.c_void_p(xh.data_ptr()), tdq.BF16 if case.x_is_bf16 else tdq.F32, 1, M, C, ctypes.byref(params),
+            ctypes.c_void_p(wcodes.data_ptr()), ctypes.c_void_p(wscale.data_ptr()), None, O,
+            ctypes.c_void_p(yh.data_ptr()), tdq.F32, ctypes.c_void_p(xs[0].data_ptr()),
+            ctypes.c_void_p(codes[0].data_ptr()), ctypes.c_void_p(scales[0].data_ptr()),
+            ctypes.c_void_p(ys[0].data_ptr()), ctypes.c_void_p(wsp.data_ptr()), wsp.numel(), ctypes.c_void_p(stream))
+        if rc != tdq.OK:
+            raise RuntimeError("tdq_quant_linear_host: " + tdq.status_string(rc))
+
+    e2e_steps = max(2, min(args.steps, 5))
+    e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+
+    times = torch.tensor([total_ms, q_ms, l_ms, e2e_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    total_ms, q_ms, l_ms, e2e_ms = [float(v) for v in times.tolist()]
+
+    if rank == 0:
+        peaks = load_peaks()
+        K = args.steps
+        qb, lb = quant_bytes(M, C, esize), linear_bytes(M, C, O)
+        ops = 2.0 * M * C * O
+        q_gbs = qb * K / (q_ms * 1e-3) / 1e9
+        l_gbs = lb * K / (l_ms * 1e-3) / 1e9
+        l_tops = ops * K / (l_ms * 1e-3) / 1e12
+        int8_peak = 2.0 * peaks["bf16_tflops"]            # nominal int8 : bf16 ratio on the measured bf16 peak
+        q_kernel = dict(name="tdq_quantize_act", ms=q_ms / K, gbs=q_gbs, frac_hbm=q_gbs / peaks["hbm_gbs"],
+                        frac_hbm_8tbs=q_gbs / 8000.0, algorithmic_bytes=qb)
+        l_kernel = dict(name="tdq_w4a4_linear", ms=l_ms / K, tops=l_tops, frac_int8=l_tops / int8_peak,
+                        frac_int8_4500=l_tops / 4500.0, gbs=l_gbs, frac_hbm=l_gbs / peaks["hbm_gbs"],
+                        algorithmic_bytes=lb, ops=ops,
+                        bound="hbm" if lb / peaks["hbm_gbs"] / 1e9 > ops / int8_peak / 1e12 else "tensor")
+        if l_ms >= q_ms:
+            if l_kernel["bound"] == "hbm":
+                roof = dict(kernel="tdq_w4a4_linear", bound="hbm", achieved=l_gbs, peak=peaks["hbm_gbs"],
+                            unit="GB/s", frac=l_gbs / peaks["hbm_gbs"], traffic=None)
+            else:
+                roof = dict(kernel="tdq_w4a4_linear", bound="tensor", achieved=l_tops, peak=int8_peak,
+                            unit="TOP/s", frac=l_tops / int8_peak, traffic=None)
+        else:
+            roof = dict(kernel="tdq_quantize_act", bound="hbm", achieved=q_gbs, peak=peaks["hbm_gbs"], unit="GB/s",
+                        frac=q_gbs / peaks["hbm_gbs"], traffic=None)
+        roof["peak_source"] = peaks["source"]
+        e2e_value = world * qb * e2e_steps / (e2e_ms * 1e-3) / 1e9
+        out = dict(metric=METRIC, value=world * q_gbs, unit="GB/s", n_gpus=world, steps=K, warmup=args.warmup,
+                   ms_per_step=total_ms / K, higher_is_better=True, scaling="weak", vs_baseline=None,
+                   dtype="f32 quantizer arithmetic on bf16 input / int8 x int8 -> int32 tensor-core contraction / f32 scaling",
+                   data="synthetic",
+                   config=dict(workload=case.name, x=[int(v) for v in case.x.shape], w=[int(v) for v in case.w.shape],
+                               g=32, tau=1.0, zr=0.2, y_dtype="f32",
+                               cache="rotating %d buffer sets, %.0f MB per step (L2 is 126 MB)" % (nsets, step_bytes / 1e6),
+                               parallelism="rows sharded, %d replica(s)" % world),
+                   kernels=dict(quantize_act=q_kernel, w4a4_linear=l_kernel,
+                                step_tokens_per_s=world * M * K / (total_ms * 1e-3)),
+                   roofline=roof, clocks=clocks, gpu_launches=int(launches),
+                   e2e=dict(value=e2e_value, unit="GB/s", ms_per_step=e2e_ms / e2e_steps,
+                            h2d_bytes_per_step=int(M * C * esize), d2h_bytes_per_step=int(M * O * 4),
+                            api="tdq_quant_linear_host"))
+        if world == 1 and not args.no_cpu_baseline:
+            leg = cpu_oracle_leg(case, min(M, args.cpu_rows))
+            out["cpu_baseline"] = dict(value=leg["quant_gbs"], unit="GB/s", cores=leg["cores"], kind="oracle",
+                                       sample="first %d of %d token rows of %s, quantizer then linear, once"
+                                              % (leg["rows"], M, case.name),
+                                       linear_tops=leg["linear_tops"], quant_s=leg["quant_s"],
+                                       linear_s=leg["linear_s"])
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="tdq", choices=["tdq", "reference"])
+    ap.add_argument("--workload", default="cfg4", choices=["cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--cpu-rows", type=int, default=18464)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        args.warmup = max(args.warmup, 3)
+        run_tdq(args)
+
+
+if __name__ == "__main__":
+    main()

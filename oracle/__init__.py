@@ -51,7 +51,7 @@ def _load():
             lib.tdq_oracle_quantize_act.restype = ctypes.c_int
             lib.tdq_oracle_quantize_weight.argtypes = [vp, ctypes.c_int, i64, i64, i32, vp, vp, vp]
             lib.tdq_oracle_quantize_weight.restype = ctypes.c_int
-            lib.tdq_oracle_w4a4_linear.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, i32, vp, vp, vp]
+            lib.tdq_oracle_w4a4_linear.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, i32, vp, vp, vp, vp]
             lib.tdq_oracle_w4a4_linear.restype = ctypes.c_int
             lib.tdq_oracle_num_threads.restype = ctypes.c_int
             _lib = lib
@@ -123,7 +123,8 @@ def quantize_weight(w, pad_to=32):
 def w4a4_linear(xcodes, xscale, wcodes, wscale, bias=None, g=32, want_acc=False):
     """Algorithm S1 step 10 as an integer contraction plus scaling.
 
-    Returns dict y float32 [M, O], y_d float64 [M, O] and, when asked, acc int32 [M, O, K].
+    Returns dict y float32 [M, O], y_d float64 [M, O], t_abs float64 [M, O] (size of the summed
+    terms, s_o * sum_k Delta_k |acc_k|) and, when asked, acc int32 [M, O, K].
     """
     xcodes = np.ascontiguousarray(xcodes, np.uint8)
     wcodes = np.ascontiguousarray(wcodes, np.uint8)
@@ -135,11 +136,12 @@ def w4a4_linear(xcodes, xscale, wcodes, wscale, bias=None, g=32, want_acc=False)
     O = wcodes.shape[0]
     K = I_pad // g
     assert wcodes.shape[1] == half and xscale.shape == (M, K) and wscale.shape == (O,)
-    out = dict(y=np.empty((M, O), np.float32), y_d=np.empty((M, O), np.float64))
+    out = dict(y=np.empty((M, O), np.float32), y_d=np.empty((M, O), np.float64),
+               t_abs=np.empty((M, O), np.float64))
     acc = np.empty((M, O, K), np.int32) if want_acc else None
     rc = _load().tdq_oracle_w4a4_linear(_ptr(xcodes), _ptr(xscale), _ptr(wcodes), _ptr(wscale),
                                         _ptr(bias), M, I_pad, O, g, _ptr(out["y"]), _ptr(out["y_d"]),
-                                        _ptr(acc))
+                                        _ptr(acc), _ptr(out["t_abs"]))
     if rc != 0:
         raise ValueError("tdq_oracle_w4a4_linear rejected its arguments")
     if want_acc:

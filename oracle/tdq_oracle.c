@@ -236,11 +236,14 @@ static int unpack_code(const uint8_t* codes, int64_t idx) {
  *   acc [M, O, K] int32 (may be NULL): integer dot product of group k
  *   y_d [M, O] double (may be NULL):   s_o * sum_k Delta[m,k] * acc[m,o,k] (+ bias)
  *   y   [M, O] float  (may be NULL):   y_d rounded to binary32
+ *   t_abs [M, O] double (may be NULL): s_o * sum_k Delta[m,k] * |acc[m,o,k]|, the size of
+ *                the terms that are summed (a diagnostic for tolerances under cancellation;
+ *                not part of the method)
  */
 int tdq_oracle_w4a4_linear(const uint8_t* xcodes, const float* xscale,
                            const uint8_t* wcodes, const float* wscale,
                            const float* bias, int64_t M, int64_t I_pad, int64_t O,
-                           int32_t g, float* y, double* y_d, int32_t* acc) {
+                           int32_t g, float* y, double* y_d, int32_t* acc, double* t_abs) {
     if (!xcodes || !xscale || !wcodes || !wscale || g <= 0 || I_pad % g) return -1;
     const int64_t K = I_pad / g;
     /* unpack every weight code once; each token row is unpacked once below. */
@@ -254,14 +257,16 @@ int tdq_oracle_w4a4_linear(const uint8_t* xcodes, const float* xscale,
         if (!xq) { status = -1; continue; }
         for (int64_t j = 0; j < I_pad; ++j) xq[j] = (int8_t)unpack_code(xcodes, m * I_pad + j);
         for (int64_t o = 0; o < O; ++o) {
-            double sum = 0.0;
+            double sum = 0.0, sum_abs = 0.0;
             for (int64_t k = 0; k < K; ++k) {
                 int32_t a = 0;
                 for (int32_t i = 0; i < g; ++i)
                     a += (int32_t)xq[k * g + i] * (int32_t)wq[o * I_pad + k * g + i];
                 if (acc) acc[(m * O + o) * K + k] = a;
                 sum += (double)xscale[m * K + k] * (double)a;
+                sum_abs += (double)xscale[m * K + k] * (double)abs(a);
             }
+            if (t_abs) t_abs[m * O + o] = (double)wscale[o] * sum_abs;
             double v = (double)wscale[o] * sum;
             if (bias) v += (double)bias[o];
             if (y_d) y_d[m * O + o] = v;

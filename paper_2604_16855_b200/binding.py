@@ -131,6 +131,8 @@ def quantize_act(x: torch.Tensor, params: ActParams | None = None, *, codes=None
         codes = torch.empty((M, K * g // 2), dtype=torch.uint8, device=x.device)
     if scale is None:
         scale = torch.empty((M, K), dtype=torch.float32, device=x.device)
+    if M == 0:          # nothing to do; an empty tensor has no device pointer to pass
+        return codes, scale
     stride = x2.stride(0) if M > 1 else C
     _check(_lib.tdq_quantize_act(_ptr(x2), _dtype_id(x2), 1, M, C, stride, ctypes.byref(p), _ptr(codes),
                                  _ptr(scale), _ptr(offset), _stream(x)), "tdq_quantize_act")

@@ -239,18 +239,18 @@ __global__ void __launch_bounds__(kFastThreads) act_g32_kernel(ActArgs a) {
 #define TDQ_CE(i, j) { __nv_bfloat162 lo_ = __hmin2(s[i], s[j]); s[j] = __hmax2(s[i], s[j]); s[i] = lo_; }
 #include "sort16_network.inc"
 #undef TDQ_CE
-            // low lanes: sorted even channels, high lanes: sorted odd channels.  The KZR-th
-            // smallest of the union is max_i min(E[i], O[KZR-1-i]); one packed min with the
-            // halves of the partner swapped covers index i and its mirror at once.
+            // low lanes: sorted even channels E, high lanes: sorted odd channels O.  The KZR-th
+            // smallest of the union is max over i + j = KZR - 1 of min(E[i], O[j]), where an
+            // index past the end counts as +inf (so for KZR > 16 the terms E[KZR-17] and
+            // O[KZR-17] stand alone).  One packed min with the partner's halves swapped covers
+            // index i and its mirror at once.
             constexpr int lo_i = (KZR > 16) ? KZR - 16 : 0;
             constexpr int hi_i = (KZR - 1 < 15) ? KZR - 1 : 15;
             constexpr int mid_i = (lo_i + hi_i) / 2;
-            __nv_bfloat162 r;
+            __nv_bfloat162 r = (KZR > 16) ? s[(KZR > 16) ? KZR - 17 : 0] : __float2bfloat162_rn(0.0f);
 #pragma unroll
-            for (int i = lo_i; i <= mid_i; ++i) {
-                __nv_bfloat162 pm = __hmin2(s[i], __lowhigh2highlow(s[KZR - 1 - i]));
-                r = (i == lo_i) ? pm : __hmax2(r, pm);
-            }
+            for (int i = lo_i; i <= mid_i && i <= hi_i; ++i)
+                r = __hmax2(r, __hmin2(s[i], __lowhigh2highlow(s[KZR - 1 - i])));
             thr = fmaxf(__low2float(r), __high2float(r));
         }
     } else {
@@ -271,7 +271,7 @@ __global__ void __launch_bounds__(kFastThreads) act_g32_kernel(ActArgs a) {
 #undef TDQ_CE
             constexpr int lo_i = (KZR > 16) ? KZR - 16 : 0;
             constexpr int hi_i = (KZR - 1 < 15) ? KZR - 1 : 15;
-            float r = 0.0f;
+            float r = (KZR > 16) ? fmaxf(s[(KZR > 16) ? KZR - 17 : 0], s[(KZR > 16) ? KZR - 1 : 16]) : 0.0f;
 #pragma unroll
             for (int i = lo_i; i <= hi_i; ++i) r = fmaxf(r, fminf(s[i], s[16 + KZR - 1 - i]));
             thr = r;

@@ -312,6 +312,8 @@ def test_linear_equals_float64_product_of_dequantized_operands(C, O, g):
                     wq["q"].reshape(O, K, g).astype(np.int64))
     np.testing.assert_array_equal(out["acc"], acc.astype(np.int32))
     assert np.abs(out["acc"]).max() <= g * 7 * 8
+    t_abs = (np.abs(acc) * xa["scale"].astype(np.float64)[:, None, :]).sum(-1) * wq["scale"].astype(np.float64)
+    np.testing.assert_allclose(out["t_abs"], t_abs, rtol=1e-12)
     # a transposed or mis-indexed weight would break this asymmetric check
     nb = oracle.w4a4_linear(xa["codes"], xa["scale"], wq["codes"], wq["scale"], g=g)
     np.testing.assert_allclose(nb["y_d"], want - bias, rtol=0, atol=float(1e-12 * scale_ref.max()))
