@@ -6,9 +6,18 @@ linear layer, as a C-ABI CUDA library (``libtdq.so``) with a thin ctypes binding
     wcodes, wscale = tdq.quantize_weight(w)
     y = tdq.w4a4_linear(codes, scale, wcodes, wscale)
 
-Importing the package loads the library and fails if it has not been built
-(``python -m paper_2604_16855_b200.build``).  There is no CPU or PyTorch fallback.
+``tdq`` (the binding module) is loaded on first access and fails if the library has not been
+built (``python -m paper_2604_16855_b200.build``).  There is no CPU or PyTorch fallback.  The
+``build`` submodule imports without the library, so that it can create it.
 """
-from . import binding as tdq  # noqa: F401
+import importlib
 
 __all__ = ["tdq"]
+
+
+def __getattr__(name):
+    if name == "tdq":
+        mod = importlib.import_module(".binding", __name__)
+        globals()["tdq"] = mod
+        return mod
+    raise AttributeError("module %r has no attribute %r" % (__name__, name))

@@ -49,7 +49,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     with ThreadPoolExecutor(max_workers=len(SOURCES)) as ex:
         objs = list(ex.map(compile_one, SOURCES))
     tmp = LIB + ".tmp.%d" % os.getpid()
-    subprocess.check_call([NVCC, "-shared", "-o", tmp] + objs + ["-cudart", "static"])
+    subprocess.check_call([NVCC, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", tmp] + objs +
+                          ["-cudart", "static"])
     os.replace(tmp, LIB)
     return LIB
 

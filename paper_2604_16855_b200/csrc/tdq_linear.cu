@@ -361,6 +361,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_linear_kernel(LinArgs a) {
         // all MMAs this CTA issued have completed unless a wait gave up; in that case give the
         // tensor core a moment before the columns are handed back
         if (sm->abort_flag) __nanosleep(1000000);
+        __syncwarp();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
 }
