@@ -1,88 +1,116 @@
 // tdq_w4a4_linear: W4A4 linear layer on the 5th-generation tensor cores (Algorithm S1 step 10).
 //
-//   acc[m,o,k] = sum_{i in group k} q_x[m,i] q_w[o,i]      tcgen05.mma kind::i8, int32 in TMEM
+//   acc[m,o,k] = sum_{i in group k} q_x[m,i] q_w[o,i]      tcgen05.mma, exact, accumulator in TMEM
 //   y[m,o]     = s_o * sum_k Delta[m,k] * acc[m,o,k] + b_o  fp32 in registers
 //
-// The activation scale changes every g codes along the contraction axis, so an int32
-// accumulator may only span one token-group.  Each group gets its own TMEM slot (a fresh
-// accumulation; groups wider than 32 codes chain g/32 instructions into the same slot), is
-// read back with tcgen05.ld, converted, multiplied by its Delta and added to a float
-// accumulator that stays in registers for the whole contraction ("promotion").
+// The activation scale changes every g codes along the contraction axis, so one tensor-core
+// accumulator may only span one token-group.  Each group gets a fresh TMEM slot (groups wider
+// than 32 codes chain g/32 instructions into it), is read back with tcgen05.ld, multiplied by
+// its Delta and added to a float accumulator that stays in registers for the whole
+// contraction ("promotion").  At g = 32 the promotion, not the tensor pipe, sets the pace: one
+// 128 x 128 x 32 instruction takes 64 clocks, while 16384 fp32 FMAs take 128 clocks of the SM's
+// FMA pipes.  The operand encoding is chosen so that nothing else is added to that:
 //
-// One persistent CTA per SM walks over 128 x 128 output tiles.  Warp roles:
-//   warps 0-7   promotion + epilogue: warp w owns TMEM lanes 32 (w % 4) .. +31 (its rows) and
-//               columns 64 (w / 4) .. +63; a thread keeps 64 float accumulators of one row.
-//   warp  8     one lane issues the MMAs and the commits that release buffers.
-//   warps 9-11  operand producers: 128-bit loads of packed codes, unpack to int8, store in
-//               the tensor core's shared-memory layout, publish with an mbarrier.
-// Two rings decouple the roles: kStages operand stages (one K-step of 32 codes each) and
-// kSlots TMEM accumulator slots, each with a full and an empty mbarrier.
+//   * g = 32: kind::f8f6f4, E4M3 operands, fp32 accumulator.  A code q in [-8, 8] is stored as
+//     the byte sign(q) << 7 | |q|, which E4M3 reads as q * 2^-9 (the values are subnormal, or
+//     2^-6 for |q| = 8).  One instruction contracts one group into a fresh slot; the 32
+//     products (|p| <= 64) and their sum (<= 1792) are exact in the fp32 accumulator, so TMEM
+//     holds acc * 2^-18 exactly and the promotion needs no integer-to-float conversion: one
+//     packed fp32 FMA per two values.
+//   * g > 32: kind::i8, int32 accumulator (several instructions chain into one slot, so the
+//     sum stays in integers; promotion is rarer).  A code is stored as the two's complement
+//     byte 16 q; TMEM holds 256 acc.
+//   The power of two is folded into the output-channel scale in the epilogue; both routes
+//   give bit-identical integer sums and the same float sequence.
 //
-// Operands.  A nibble is moved to the HIGH half of its byte, which is the two's complement
-// byte 16 q: no sign extension is needed, the integer result is 256 acc (exactly;
-// |256 acc| < 2^31 for g <= 4096) and the factor 1/256 is folded into Delta, an exact
-// power-of-two scaling.  Even channels fill the first 16 bytes of a row and odd channels the
-// second 16; both operands use the same order, so the sum is unchanged.
+// Two kernels per call:
+//   1. expand_kernel   rewrites the packed nibbles of both operands as operand bytes, in 128-row
+//      x 32-code blocks laid out in the tensor core's K-major core-matrix order (8 rows x 16
+//      bytes contiguous), and regroups the activation scales as [row block][group][128 rows].
+//      The blocks live in the caller's workspace; a block is one contiguous piece, so the GEMM
+//      moves operands with plain 1-D bulk copies (cp.async.bulk + mbarrier) and no tensor maps.
+//   2. w4a4_gemm_kernel   persistent, one CTA per SM, 128 x 128 output tiles.  Warp roles:
+//        warps 0-1   producers: one lane each issues the bulk copies of alternate ring stages
+//        warp  2     one lane issues the MMAs and the commits that release buffers
+//        warps 4-11  promotion + epilogue: warp w owns TMEM lanes 32 (w % 4).. (its rows) and 64
+//                    columns; a thread keeps 64 float accumulators of one output row
+//      The promotion warps take most of the register file (setmaxnreg): a thread holds its 64
+//      accumulators plus two 32-value landing buffers, so that one TMEM load is in flight while
+//      the FMAs on the other buffer issue.
+//      A work item is one 128-row block of A with a range of column tiles.  The item's scales,
+//      and its A block when the whole K extent fits, are loaded once per item; B (and A
+//      otherwise) streams through a ring of stages of 4 K-steps.  TMEM holds four 128-column
+//      accumulator slots, each with a full/empty mbarrier pair.
+//      In the epilogue every thread parks its 64 outputs in its own shared-memory strip; the
+//      promotion warps then read the tile back row by row, so that one warp instruction stores
+//      512 contiguous bytes of y.
 //
-// Shared-memory operand layout: K-major, no swizzle.  A 32-byte row splits into two 16-byte
-// chunks; 8 rows x 16 bytes form one contiguous 128-byte core matrix; the two K-chunks of an
-// 8-row band are 128 bytes apart (leading byte offset), bands are 256 bytes apart (stride
-// byte offset).
-//
-// Every wait on an mbarrier is bounded: after about a second the thread records a code in
-// the workspace status word and raises a CTA-wide flag; every role then leaves its loops,
-// the CTA releases its TMEM and returns.
+// Every wait on an mbarrier is bounded: after about a second the thread records a code in the
+// workspace status word and raises a CTA-wide flag; every role then leaves its loops, the CTA
+// releases its TMEM and returns.
 #include "tdq_common.cuh"
 
 namespace tdq {
 namespace {
 
-constexpr int kBM = 128;              // rows per tile = TMEM lanes
-constexpr int kBN = 128;              // columns per tile = one TMEM slot
-constexpr int kStages = 8;            // operand ring, one K-step (32 codes) per stage
-constexpr int kSlots = 4;             // TMEM accumulator ring (4 x 128 = 512 columns)
+constexpr int kBM = 128;                 // rows per tile = TMEM lanes
+constexpr int kBN = 128;                 // columns per tile = one TMEM slot
+constexpr int kSlots = 4;                // TMEM accumulator ring (4 x 128 = 512 columns)
+constexpr int kChunk = 4;                // K-steps (of 32 codes) per ring stage
+constexpr int kBlock = 128 * 32;         // operand bytes of one 128-row block and one K-step
+constexpr int kScaleBlock = 128 * 4;     // the scales of one 128-row block and one group
+constexpr int kMaxStages = 8;
+constexpr int kProdWarps = 2;
+constexpr int kMmaWarp = 2;
+constexpr int kPromoWarp0 = 4;
 constexpr int kPromoWarps = 8;
-constexpr int kMmaWarp = 8;
-constexpr int kProdWarp0 = 9;
-constexpr int kProdWarps = 3;
-constexpr int kThreads = (kPromoWarps + 1 + kProdWarps) * 32;   // 384: 12 warps leave 168 registers per thread
-constexpr int kProdThreads = kProdWarps * 32;
-constexpr int kJobs = (kBM + kBN + kProdThreads - 1) / kProdThreads;   // operand rows per producer thread
-constexpr int kABytes = kBM * 32, kBBytes = kBN * 32;
-static_assert(kABytes == kBBytes, "the producers address both operand rings with one stage stride");
+constexpr int kThreads = (kPromoWarp0 + kPromoWarps) * 32;   // 384
+constexpr int kStripBytes = 256;         // one thread's 64 fp32 outputs (128 bytes used for bf16)
+constexpr int kStagingBytes = kPromoWarps * 32 * kStripBytes;
+constexpr int kWsbBytes = kPromoWarps * 512;   // per warp: 64 output-channel scales and 64 biases
+constexpr int kCtrlBytes = 256;
+constexpr int kSmemLimit = 232448;       // 227 KB per CTA
 constexpr uint32_t kTmemCols = kSlots * kBN;
 constexpr long long kTimeoutCycles = 2000000000LL;
-// S32 accumulator, signed 8-bit A and B, both K-major, N = 128, M = 128
-constexpr uint32_t kIdesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) |
-                            ((uint32_t)(kBM >> 4) << 24);
+constexpr int kExpandThreads = 512;
+constexpr int kRegsControl = 40, kRegsPromo = 232;   // 128 * 40 + 256 * 232 = 384 * 168
+
+// instruction descriptors: M = 128, N = 128, both operands K-major
+constexpr uint32_t kIdescShape = ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+constexpr uint32_t kIdescI8 = (2u << 4) | (1u << 7) | (1u << 10) | kIdescShape;   // S32 += S8 * S8
+constexpr uint32_t kIdescF8 = (1u << 4) | (0u << 7) | (0u << 10) | kIdescShape;   // F32 += E4M3 * E4M3
 
 struct LinArgs {
-    const uint8_t* xcodes;
-    const float* xscale;
-    const uint8_t* wcodes;
+    const uint8_t* a_blocks;   // [tiles_m][n_steps] operand blocks
+    const uint8_t* b_blocks;   // [tiles_n][n_steps] operand blocks
+    const uint8_t* s_blocks;   // [tiles_m][Kg] scale blocks
     const float* wscale;
     const float* bias;
     int64_t M, O;
-    int32_t row_bytes;      // I_pad / 2
-    int32_t n_steps;        // I_pad / 32
-    int32_t steps_per_grp;  // g / 32
-    int32_t Kg;             // groups per token
-    int32_t tiles_m, tiles_n;
+    int32_t n_steps;           // I_pad / 32
+    int32_t steps_per_grp;     // g / 32
+    int32_t Kg;                // groups per token
+    int32_t tiles_m, tiles_n, n_parts;
+    int32_t a_resident;        // the item's whole A block stays in shared memory
+    int32_t n_stages;
+    uint32_t ares_off, ring_off, stage_bytes, staging_off, wsb_off;   // shared-memory carve-up
     void* y;
     int64_t y_stride;
     int32_t* acc_debug;
     uint32_t* status;
-    int32_t vec_ok;         // y, wscale, bias 16-byte aligned and y_stride % 4 == 0: float4 epilogue
+    int32_t vec_ok;            // y rows can be written with 16-byte aligned vector stores
+    float out_scale;           // 2^18 (E4M3 route) or 2^-8 (int8 route)
 };
 
-struct __align__(128) Smem {
-    uint8_t a[kStages][kABytes];
-    uint8_t b[kStages][kBBytes];
-    uint64_t full[kStages], empty[kStages];
+struct Ctrl {
+    uint64_t full[kMaxStages], empty[kMaxStages];
     uint64_t tfull[kSlots], tempty[kSlots];
+    uint64_t a_full, a_empty;
+    uint64_t strips_ready, strips_free;   // epilogue hand-over between the promotion warps
     uint32_t tmem_base;
     volatile int abort_flag;
 };
+static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block outgrew its reservation");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -90,8 +118,8 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
 }
 
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
 
 __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
@@ -106,38 +134,95 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Bounded wait: false when the phase did not complete within the time limit or another
-// role of this CTA already gave up.  `code` names the wait in the status word.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Smem* sm, uint32_t* status, uint32_t code) {
-    if (mbar_test(bar, parity)) return true;
-    const long long t0 = clock64();
-    for (;;) {
-#pragma unroll 1
-        for (int i = 0; i < 32; ++i)
-            if (mbar_test(bar, parity)) return true;
-        if (sm->abort_flag) return false;
-        if (clock64() - t0 > kTimeoutCycles) {
-            atomicCAS(status, 0u, code | ((uint32_t)blockIdx.x << 8));
-            sm->abort_flag = 1;
-            return false;
-        }
-    }
+__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;   // try_wait may suspend the thread for a short, hardware-chosen time before it answers
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
 }
 
-__device__ __forceinline__ uint64_t smem_desc_kmajor_noswizzle(uint32_t saddr) {
-    // start address, leading byte offset 128, stride byte offset 256 (all >> 4), version 1
+// Slow path of a bounded wait: polls until the phase completes, another role of this CTA has
+// given up, or about a second has passed; then it records which wait gave up (first writer
+// wins) and raises the CTA-wide flag.
+__device__ __forceinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, Ctrl* c, uint32_t* status, uint32_t code) {
+    long long t0 = 0;
+    uint32_t polls = 0;
+#pragma unroll 1
+    while (!mbar_try(bar, parity)) {
+        if ((++polls & 63u) == 0u) {
+            if (c->abort_flag) return false;
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            if (now - t0 > kTimeoutCycles) {
+                atomicCAS(status, 0u, code | ((uint32_t)blockIdx.x << 8));
+                c->abort_flag = 1;
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+// Bounded wait by one thread: false when the phase did not complete in time.  `code` names the
+// wait in the status word.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Ctrl* c, uint32_t* status, uint32_t code) {
+    if (mbar_test(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, c, status, code);
+}
+
+// Bounded wait by a converged warp; the answer is the same in every lane.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, Ctrl* c, uint32_t* status, uint32_t code) {
+    if (__all_sync(0xffffffffu, mbar_test(bar, parity))) return true;
+    return __all_sync(0xffffffffu, mbar_wait_slow(bar, parity, c, status, code));
+}
+
+// lane 0 of a converged warp arrives; predicated, so the warp does not diverge
+__device__ __forceinline__ void mbar_arrive_lane0(uint64_t* bar, int lane) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.eq.s32 p, %1, 0;\n\t"
+        "@p mbarrier.arrive.shared::cta.b64 _, [%0];\n\t}"
+        ::"r"(smem_u32(bar)), "r"(lane)
+        : "memory");
+}
+
+// global -> shared bulk copy that reports its bytes to an mbarrier
+__device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+
+// K-major, no swizzle: 8 rows x 16 bytes are one contiguous 128-byte core matrix; the two
+// K-halves of an 8-row band are 128 bytes apart (leading byte offset) and bands are 256 bytes
+// apart (stride byte offset).  Offsets are stored >> 4; bit 46 is the descriptor version.
+// The start address sits in the low 14 bits, so adding (bytes >> 4) moves the descriptor.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr) {
     return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(128 >> 4) << 16) | ((uint64_t)(256 >> 4) << 32) |
            (1ull << 46);
 }
 
-__device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                       uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
+template <bool I8>
+__device__ __forceinline__ void mma_issue(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+    if (I8)
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(kIdescI8), "r"(accumulate)
+            : "memory");
+    else
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(kIdescF8), "r"(accumulate)
+            : "memory");
 }
 
 __device__ __forceinline__ void mma_commit(uint64_t* bar) {
@@ -145,15 +230,18 @@ __device__ __forceinline__ void mma_commit(uint64_t* bar) {
                  : "memory");
 }
 
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+// 32 consecutive columns of this warp's 32 TMEM lanes: lane i receives row i, v[j] = column j.
+// The operands are declared read-write so that a landing buffer keeps its registers for the
+// whole kernel (pure outputs would be renamed at every load and copied at every loop edge).
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* v) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
         "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
         "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]),
+          "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15]),
+          "+r"(v[16]), "+r"(v[17]), "+r"(v[18]), "+r"(v[19]), "+r"(v[20]), "+r"(v[21]), "+r"(v[22]), "+r"(v[23]),
+          "+r"(v[24]), "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]), "+r"(v[30]), "+r"(v[31])
         : "r"(taddr)
         : "memory");
 }
@@ -161,32 +249,152 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-// 16 packed bytes (32 codes) -> two 16-byte chunks of bytes 16*q: even channels, odd channels.
-__device__ __forceinline__ void unpack16(const uint4 p, uint4& even, uint4& odd) {
-    even = make_uint4((p.x << 4) & 0xF0F0F0F0u, (p.y << 4) & 0xF0F0F0F0u, (p.z << 4) & 0xF0F0F0F0u,
-                      (p.w << 4) & 0xF0F0F0F0u);
-    odd = make_uint4(p.x & 0xF0F0F0F0u, p.y & 0xF0F0F0F0u, p.z & 0xF0F0F0F0u, p.w & 0xF0F0F0F0u);
+__device__ __forceinline__ uint64_t pack2(uint32_t lo, uint32_t hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t p, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(p));
+}
+// acc = v * d + acc on two packed floats
+__device__ __forceinline__ void fma2(uint64_t& acc, uint64_t v, uint64_t d) {
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(v), "l"(d));
 }
 
-// byte offset of row r, K-chunk 0 inside one K-step's operand block (see the layout note above)
-__device__ __forceinline__ uint32_t row_off(int r) { return (uint32_t)((r >> 3) * 256 + (r & 7) * 16); }
+// shared memory by 32-bit shared-window address
+__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) {
+    asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ void sts64(uint32_t addr, uint32_t x, uint32_t y) {
+    asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(addr), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
 
-template <bool YBF16>
-__global__ void __launch_bounds__(kThreads, 1) w4a4_linear_kernel(LinArgs a) {
+template <int N>
+__device__ __forceinline__ void setmaxnreg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N>
+__device__ __forceinline__ void setmaxnreg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+
+// ------------------------------------------------------------------------------------------
+// kernel 1: nibbles -> operand bytes in core-matrix order, scales regrouped by row block
+
+// four two's complement bytes 16 q -> four sign-magnitude bytes (q < 0) << 7 | |q|
+__device__ __forceinline__ uint32_t to_sign_magnitude(uint32_t b16) {
+    uint32_t neg;   // 0xFF where the byte is negative: prmt with the selector's replicate-sign bit set
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(neg) : "r"(b16), "r"(0u), "r"(0xBA98u));
+    const uint32_t abs16 = (b16 ^ neg) + (neg & 0x01010101u);             // 16 |q| per byte, no carry leaves a byte
+    return (abs16 >> 4) | (neg & 0x80808080u);
+}
+
+// 8 packed codes (even channel in the low nibble) -> 8 operand bytes in channel order
+template <bool I8>
+__device__ __forceinline__ void expand8(uint32_t p, uint32_t& lo, uint32_t& hi) {
+    uint32_t ev = (p << 4) & 0xF0F0F0F0u;   // channels 0,2,4,6 as bytes 16 q
+    uint32_t od = p & 0xF0F0F0F0u;          // channels 1,3,5,7
+    if (!I8) {
+        ev = to_sign_magnitude(ev);
+        od = to_sign_magnitude(od);
+    }
+    lo = __byte_perm(ev, od, 0x5140u);
+    hi = __byte_perm(ev, od, 0x7362u);
+}
+
+struct ExpandArgs {
+    const uint8_t* xcodes;
+    const float* xscale;
+    const uint8_t* wcodes;
+    uint8_t* a_blocks;
+    uint8_t* b_blocks;
+    uint8_t* s_blocks;
+    int64_t M, O;
+    int32_t row_bytes;       // I_pad / 2
+    int32_t n_steps, n_chunks, steps_per_grp, Kg;
+    int32_t tiles_m, tiles_n;
+};
+
+// One CTA rewrites one (128-row block, 4 K-steps) piece: thread t takes row t / 4 and K-step t % 4.
+template <bool I8>
+__global__ void __launch_bounds__(kExpandThreads) expand_kernel(ExpandArgs a) {
+    const int piece = blockIdx.x;
+    const int blk = piece / a.n_chunks, kc = piece % a.n_chunks;
+    const int r = threadIdx.x >> 2;
+    const int ks = kc * kChunk + (threadIdx.x & 3);
+    if (ks >= a.n_steps) return;
+    const bool is_a = blk < a.tiles_m;
+    const int tile = is_a ? blk : blk - a.tiles_m;
+    const int64_t row = (int64_t)tile * 128 + r;
+    const int64_t rows = is_a ? a.M : a.O;
+    const uint8_t* src = is_a ? a.xcodes : a.wcodes;
+    uint4 p = make_uint4(0, 0, 0, 0);
+    if (row < rows) p = __ldg(reinterpret_cast<const uint4*>(src + row * a.row_bytes + (int64_t)ks * 16));
+    uint4 c0, c1;
+    expand8<I8>(p.x, c0.x, c0.y);
+    expand8<I8>(p.y, c0.z, c0.w);
+    expand8<I8>(p.z, c1.x, c1.y);
+    expand8<I8>(p.w, c1.z, c1.w);
+    uint8_t* dst = (is_a ? a.a_blocks : a.b_blocks) + ((int64_t)tile * a.n_steps + ks) * kBlock;
+    const int off = (r >> 3) * 256 + (r & 7) * 16;
+    *reinterpret_cast<uint4*>(dst + off) = c0;
+    *reinterpret_cast<uint4*>(dst + off + 128) = c1;
+    if (is_a && ks % a.steps_per_grp == 0) {
+        const int grp = ks / a.steps_per_grp;
+        float s = 0.0f;
+        if (row < rows) s = __ldg(a.xscale + row * a.Kg + grp);
+        reinterpret_cast<float*>(a.s_blocks + ((int64_t)tile * a.Kg + grp) * kScaleBlock)[r] = s;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// kernel 2: the GEMM
+
+// Test-only dump of 32 integer group sums of one output row (the debug instantiation of the kernel).
+template <bool I8>
+__device__ __noinline__ void debug_store(const LinArgs& a, const uint32_t* v, int64_t m, int64_t n0, int grp) {
+#pragma unroll 1
+    for (int q = 0; q < 32; ++q)
+        if (n0 + q < a.O)
+            a.acc_debug[(m * a.O + n0 + q) * a.Kg + grp] =
+                I8 ? ((int32_t)v[q] >> 8) : __float2int_rn(__uint_as_float(v[q]) * 262144.0f);
+}
+
+template <bool I8, bool YBF16, bool DBG>
+__global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
     extern __shared__ uint8_t smem_raw[];
-    Smem* sm = reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+    uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+    Ctrl* c = reinterpret_cast<Ctrl*>(sm);
+    const uint32_t sm_s = smem_u32(sm);
+    const uint32_t scales_s = sm_s + kCtrlBytes;        // [Kg][128] floats of the item
+    const uint32_t ares_s = sm_s + a.ares_off;          // [n_steps] operand blocks of the item, if resident
+    const uint32_t ring_s = sm_s + a.ring_off;
     const int t = threadIdx.x, warp = t >> 5, lane = t & 31;
+    const bool resident = a.a_resident != 0;
 
     if (t == 0) {
-        for (int i = 0; i < kStages; ++i) { mbar_init(&sm->full[i], kProdWarps); mbar_init(&sm->empty[i], 1); }
-        for (int i = 0; i < kSlots; ++i) { mbar_init(&sm->tfull[i], 1); mbar_init(&sm->tempty[i], kPromoWarps); }
-        sm->abort_flag = 0;
+        for (int i = 0; i < kMaxStages; ++i) { mbar_init(&c->full[i], 1); mbar_init(&c->empty[i], 1); }
+        for (int i = 0; i < kSlots; ++i) { mbar_init(&c->tfull[i], 1); mbar_init(&c->tempty[i], kPromoWarps); }
+        mbar_init(&c->a_full, 1);
+        mbar_init(&c->a_empty, 1 + kPromoWarps);
+        mbar_init(&c->strips_ready, kPromoWarps);
+        mbar_init(&c->strips_free, kPromoWarps);
+        c->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == kMmaWarp) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm->tmem_base)),
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&c->tmem_base)),
                      "r"(kTmemCols)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -194,165 +402,291 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_linear_kernel(LinArgs a) {
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_base = sm->tmem_base;
-    const int64_t n_tiles = (int64_t)a.tiles_m * a.tiles_n;
-    const int grp_per_tile = a.n_steps / a.steps_per_grp;
+    const uint32_t tmem_base = c->tmem_base;
 
-    if (warp < kPromoWarps) {
-        // ------------------------------------------------------------ promotion + epilogue
-        const int row = (warp & 3) * 32 + lane;
-        const int col0 = (warp >> 2) * (kBN / 2);
-        uint32_t gc = 0;   // groups consumed so far (across tiles): slot = gc % kSlots
-        for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
-            const int64_t m = (tile / a.tiles_n) * kBM + row;
-            const int64_t n0 = (tile % a.tiles_n) * kBN + col0;
-            const bool row_ok = m < a.M;
-            const float* srow = a.xscale + (row_ok ? m : 0) * a.Kg;
-            float yacc[kBN / 2];
-#pragma unroll
-            for (int j = 0; j < kBN / 2; ++j) yacc[j] = 0.0f;
-            float d_next = row_ok ? __ldg(srow) * (1.0f / 256.0f) : 0.0f;
+    const int n_items = a.tiles_m * a.n_parts;
+    const int n_chunks = (a.n_steps + kChunk - 1) / kChunk;
+    const int spg = a.steps_per_grp;
+    auto part_begin = [&](int part) { return (int)(((int64_t)part * a.tiles_n) / a.n_parts); };
+
+    if (warp < kPromoWarp0) {
+        setmaxnreg_dec<kRegsControl>();
+        if (warp < kProdWarps && lane == 0) {
+            // ------------------------------------------------------------ producers (one lane each)
+            uint32_t sc = 0, s = 0, ph = 0, ic = 0;   // stage counter, its ring slot and phase; items so far
             bool ok = true;
-            for (int grp = 0; grp < grp_per_tile && ok; ++grp, ++gc) {
-                const float d256 = d_next;
-                if (grp + 1 < grp_per_tile) d_next = row_ok ? __ldg(srow + grp + 1) * (1.0f / 256.0f) : 0.0f;
-                const uint32_t slot = gc % kSlots;
-                ok = __all_sync(0xffffffffu, mbar_wait(&sm->tfull[slot], (gc / kSlots) & 1, sm, a.status, 2u));
-                if (!ok) break;   // warp-uniform: the TMEM loads below are warp-collective
-                tc_fence_after();
-                const uint32_t taddr = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + slot * kBN + col0;
-                uint32_t v0[32], v1[32];
-                tmem_ld32(taddr, v0);
-                tmem_ld32(taddr + 32, v1);
-                tmem_ld_wait();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&sm->tempty[slot]);   // slot may be overwritten from here on
-#pragma unroll
-                for (int j = 0; j < 32; ++j) yacc[j] = fmaf(d256, (float)(int32_t)v0[j], yacc[j]);
-#pragma unroll
-                for (int j = 0; j < 32; ++j) yacc[32 + j] = fmaf(d256, (float)(int32_t)v1[j], yacc[32 + j]);
-                if (a.acc_debug && row_ok) {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        if (n0 + j < a.O) a.acc_debug[(m * a.O + n0 + j) * a.Kg + grp] = ((int32_t)v0[j]) >> 8;
-                        if (n0 + 32 + j < a.O) a.acc_debug[(m * a.O + n0 + 32 + j) * a.Kg + grp] = ((int32_t)v1[j]) >> 8;
+            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++ic) {
+                const int mt = item / a.n_parts, part = item % a.n_parts;
+                const uint8_t* a_src = a.a_blocks + (int64_t)mt * a.n_steps * kBlock;
+                if (warp == 0) {
+                    ok = mbar_wait(&c->a_empty, (ic & 1) ^ 1, c, a.status, 1u);
+                    if (!ok) break;
+                    const uint32_t sbytes = (uint32_t)a.Kg * kScaleBlock;
+                    mbar_expect_tx(&c->a_full, sbytes + (resident ? (uint32_t)a.n_steps * kBlock : 0u));
+                    const uint8_t* s_src = a.s_blocks + (int64_t)mt * a.Kg * kScaleBlock;
+                    for (uint32_t off = 0; off < sbytes; off += 16384u)
+                        bulk_load(scales_s + off, s_src + off, min(16384u, sbytes - off), &c->a_full);
+                    if (resident)
+                        for (int kc = 0; kc < n_chunks; ++kc) {
+                            const int nk = min(kChunk, a.n_steps - kc * kChunk);
+                            bulk_load(ares_s + kc * kChunk * kBlock, a_src + (int64_t)kc * kChunk * kBlock,
+                                      (uint32_t)nk * kBlock, &c->a_full);
+                        }
+                }
+                for (int nt = part_begin(part); nt < part_begin(part + 1) && ok; ++nt) {
+                    const uint8_t* b_src = a.b_blocks + (int64_t)nt * a.n_steps * kBlock;
+                    for (int kc = 0; kc < n_chunks; ++kc, ++sc) {
+                        if ((int)(sc & 1u) == warp) {
+                            ok = mbar_wait(&c->empty[s], ph ^ 1, c, a.status, 5u);
+                            if (!ok) break;
+                            const int nk = min(kChunk, a.n_steps - kc * kChunk);
+                            const uint32_t stage = ring_s + s * a.stage_bytes;
+                            mbar_expect_tx(&c->full[s], (uint32_t)nk * kBlock * (resident ? 1u : 2u));
+                            bulk_load(stage, b_src + (int64_t)kc * kChunk * kBlock, (uint32_t)nk * kBlock, &c->full[s]);
+                            if (!resident)
+                                bulk_load(stage + kChunk * kBlock, a_src + (int64_t)kc * kChunk * kBlock,
+                                          (uint32_t)nk * kBlock, &c->full[s]);
+                        }
+                        if (++s == (uint32_t)a.n_stages) { s = 0; ph ^= 1; }
                     }
                 }
             }
-            if (!ok) break;
-            // epilogue: y = s_o * sum + bias
-            if (row_ok) {
-                if (!YBF16 && a.vec_ok && n0 + kBN / 2 <= a.O) {
-                    float* yrow = reinterpret_cast<float*>(a.y) + m * a.y_stride + n0;
-#pragma unroll
-                    for (int j = 0; j < kBN / 2; j += 4) {
-                        const float4 s4 = __ldg(reinterpret_cast<const float4*>(a.wscale + n0 + j));
-                        float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f);
-                        if (a.bias) b4 = __ldg(reinterpret_cast<const float4*>(a.bias + n0 + j));
-                        float4 o;
-                        o.x = __fmaf_rn(s4.x, yacc[j], b4.x);
-                        o.y = __fmaf_rn(s4.y, yacc[j + 1], b4.y);
-                        o.z = __fmaf_rn(s4.z, yacc[j + 2], b4.z);
-                        o.w = __fmaf_rn(s4.w, yacc[j + 3], b4.w);
-                        __stcs(reinterpret_cast<float4*>(yrow + j), o);
-                    }
-                } else {
-#pragma unroll
-                    for (int j = 0; j < kBN / 2; ++j) {
-                        const int64_t n = n0 + j;
-                        if (n < a.O) {
-                            const float b = a.bias ? __ldg(a.bias + n) : 0.0f;
-                            const float v = __fmaf_rn(__ldg(a.wscale + n), yacc[j], b);
-                            if (YBF16)
-                                reinterpret_cast<__nv_bfloat16*>(a.y)[m * a.y_stride + n] = __float2bfloat16_rn(v);
-                            else
-                                reinterpret_cast<float*>(a.y)[m * a.y_stride + n] = v;
+        } else if (warp == kMmaWarp && lane == 0) {
+            // ------------------------------------------------------------ MMA issue (one lane)
+            uint32_t s = 0, ph = 0, slot = 0, tph = 0, ic = 0;
+            const uint64_t ares_desc = smem_desc(ares_s);
+            bool ok = true;
+            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++ic) {
+                const int part = item % a.n_parts;
+                ok = mbar_wait(&c->a_full, ic & 1, c, a.status, 6u);
+                for (int nt = part_begin(part); nt < part_begin(part + 1) && ok; ++nt) {
+                    int sub = 0, kj = 0;
+                    uint64_t bdesc = 0;
+                    for (int ks = 0; ks < a.n_steps; ++ks) {
+                        if (kj == 0) {
+                            ok = mbar_wait(&c->full[s], ph, c, a.status, 4u);
+                            if (!ok) break;
+                            bdesc = smem_desc(ring_s + s * a.stage_bytes);
+                        }
+                        if (sub == 0) {
+                            ok = mbar_wait(&c->tempty[slot], tph ^ 1, c, a.status, 3u);
+                            if (!ok) break;
+                        }
+                        tc_fence_after();
+                        const uint64_t adesc = resident ? ares_desc + (uint64_t)(ks * (kBlock >> 4))
+                                                        : bdesc + (uint64_t)((kChunk + kj) * (kBlock >> 4));
+                        mma_issue<I8>(tmem_base + slot * kBN, adesc, bdesc + (uint64_t)(kj * (kBlock >> 4)),
+                                      sub == 0 ? 0u : 1u);
+                        if (++sub == spg) {
+                            sub = 0;
+                            mma_commit(&c->tfull[slot]);
+                            if (++slot == kSlots) { slot = 0; tph ^= 1; }
+                        }
+                        if (++kj == kChunk || ks == a.n_steps - 1) {
+                            kj = 0;
+                            mma_commit(&c->empty[s]);
+                            if (++s == (uint32_t)a.n_stages) { s = 0; ph ^= 1; }
                         }
                     }
                 }
-            }
-        }
-    } else if (warp == kMmaWarp) {
-        // ------------------------------------------------------------ MMA issue (one lane)
-        if (lane == 0) {
-            uint32_t it = 0, gc = 0;
-            bool ok = true;
-            for (int64_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-                for (int step = 0; step < a.n_steps && ok; ++step, ++it) {
-                    const uint32_t s = it % kStages;
-                    const int sub = step % a.steps_per_grp;
-                    const uint32_t slot = gc % kSlots;
-                    if (sub == 0) ok = mbar_wait(&sm->tempty[slot], ((gc / kSlots) & 1) ^ 1, sm, a.status, 3u);
-                    if (ok) ok = mbar_wait(&sm->full[s], (it / kStages) & 1, sm, a.status, 4u);
-                    if (!ok) break;
-                    tc_fence_after();
-                    mma_i8(tmem_base + slot * kBN, smem_desc_kmajor_noswizzle(smem_u32(sm->a[s])),
-                           smem_desc_kmajor_noswizzle(smem_u32(sm->b[s])), kIdesc, sub == 0 ? 0u : 1u);
-                    mma_commit(&sm->empty[s]);
-                    if (sub == a.steps_per_grp - 1) {
-                        mma_commit(&sm->tfull[slot]);
-                        ++gc;
-                    }
-                }
+                if (ok) mma_commit(&c->a_empty);
             }
         }
     } else {
-        // ------------------------------------------------------------ operand producers
-        // row job j: j < kBM is row j of the A tile, otherwise row j - kBM of the B tile
-        const int pt = (warp - kProdWarp0) * 32 + lane;
-        uint32_t it = 0;
-        bool ok = true;
-        for (int64_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-            const int64_t m0 = (tile / a.tiles_n) * kBM, n0 = (tile % a.tiles_n) * kBN;
-            const uint8_t* src[kJobs];
-            uint32_t dst[kJobs];
-#pragma unroll
-            for (int q = 0; q < kJobs; ++q) {
-                const int j = pt + q * kProdThreads;
-                src[q] = nullptr;
-                dst[q] = 0xffffffffu;
-                if (j < kBM) {
-                    if (m0 + j < a.M) src[q] = a.xcodes + (m0 + j) * a.row_bytes;
-                    dst[q] = row_off(j);
-                } else if (j < kBM + kBN) {
-                    if (n0 + (j - kBM) < a.O) src[q] = a.wcodes + (n0 + (j - kBM)) * a.row_bytes;
-                    dst[q] = (uint32_t)(kStages * kABytes) + row_off(j - kBM);   // b[] follows a[] in Smem
-                }
-            }
-            for (int s0 = 0; s0 < a.n_steps && ok; s0 += 4) {
-                uint4 pk[kJobs][4];
-#pragma unroll
-                for (int q = 0; q < kJobs; ++q)
-#pragma unroll
-                    for (int b = 0; b < 4; ++b) {
-                        pk[q][b] = make_uint4(0, 0, 0, 0);
-                        if (src[q] && s0 + b < a.n_steps)
-                            pk[q][b] = __ldg(reinterpret_cast<const uint4*>(src[q] + (size_t)(s0 + b) * 16));
-                    }
-#pragma unroll
-                for (int b = 0; b < 4; ++b) {
-                    if (s0 + b >= a.n_steps) break;
-                    const uint32_t s = it % kStages;
-                    ok = __all_sync(0xffffffffu, mbar_wait(&sm->empty[s], ((it / kStages) & 1) ^ 1, sm, a.status, 5u));
-                    if (!ok) break;   // warp-uniform: the warp synchronises below
-#pragma unroll
-                    for (int q = 0; q < kJobs; ++q) {
-                        if (dst[q] == 0xffffffffu) continue;
-                        uint4 ev, od;
-                        unpack16(pk[q][b], ev, od);
-                        // a[s] and b[s] blocks: stage stride is kABytes for A rows and kBBytes for B rows (equal)
-                        uint8_t* d = sm->a[0] + dst[q] + s * kABytes;
-                        *reinterpret_cast<uint4*>(d) = ev;
-                        *reinterpret_cast<uint4*>(d + 128) = od;
-                    }
-                    fence_async_smem();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&sm->full[s]);
-                    ++it;
-                }
-            }
+        setmaxnreg_inc<kRegsPromo>();
+        // ------------------------------------------------------------ promotion + epilogue
+        const int pw = warp - kPromoWarp0;
+        const int quarter = warp & 3;                 // TMEM lanes 32 * quarter .. + 31
+        const int row = quarter * 32 + lane;
+        const int col0 = (pw >> 2) * (kBN / 2);
+        const uint32_t tmem_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + col0;
+        constexpr int esz = YBF16 ? 2 : 4;
+        constexpr int kChunksPerStrip = 64 * esz / 16;             // 16-byte chunks of one strip
+        const uint32_t strips_s = sm_s + a.staging_off;
+        const uint32_t strip_s = strips_s + (uint32_t)(pw * 32 + lane) * kStripBytes;
+        const uint32_t swz = (uint32_t)lane & (kChunksPerStrip - 1);   // chunk c of a strip sits at c ^ swz
+        const uint32_t wsb_s = sm_s + a.wsb_off + (uint32_t)pw * 512;
+        const uint32_t my_scale_s = scales_s + (uint32_t)row * 4;
+
+        // groups this CTA will see, so that the next slot can be requested early
+        uint32_t total = 0;
+        for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+            const int part = item % a.n_parts;
+            total += (uint32_t)(part_begin(part + 1) - part_begin(part)) * (uint32_t)a.Kg;
         }
+
+        uint64_t yacc[kBN / 4];        // 64 floats of one output row, packed in pairs
+        uint32_t va[32], vb[32];       // landing buffers: first and second 32 columns of a slot
+#pragma unroll
+        for (int q = 0; q < 32; ++q) va[q] = vb[q] = 0u;
+        uint32_t gc = 0, slot = 0, tph = 0, ic = 0, tc = 0;   // groups, their slot and phase; items, tiles so far
+        int item = blockIdx.x, mt = 0, nt = 0, nt_end = 0, grp_left = 0;
+        uint32_t scale_s = my_scale_s;   // this row's scale of the group about to be promoted
+        int64_t m = 0, n0 = 0;
+        float w0 = 0.f, w1 = 0.f, b0 = 0.f, b1 = 0.f;   // this lane's share of the tile's channel scales and biases
+        bool ok = true, row_ok = false;
+
+        auto begin_item = [&]() {
+            mt = item / a.n_parts;
+            const int part = item % a.n_parts;
+            nt = part_begin(part);
+            nt_end = part_begin(part + 1);
+            m = (int64_t)mt * kBM + row;
+            row_ok = m < a.M;
+            ok = mbar_wait_warp(&c->a_full, ic & 1, c, a.status, 7u);
+        };
+        auto begin_tile = [&]() {
+            n0 = (int64_t)nt * kBN + col0;
+            grp_left = a.Kg;
+            scale_s = my_scale_s;
+#pragma unroll
+            for (int j = 0; j < kBN / 4; ++j) yacc[j] = 0ull;
+            const int64_t ca = n0 + lane, cb = n0 + 32 + lane;
+            w0 = ca < a.O ? __ldg(a.wscale + ca) : 0.f;
+            w1 = cb < a.O ? __ldg(a.wscale + cb) : 0.f;
+            b0 = (a.bias && ca < a.O) ? __ldg(a.bias + ca) : 0.f;
+            b1 = (a.bias && cb < a.O) ? __ldg(a.bias + cb) : 0.f;
+        };
+        // y = (s_o * 2^e) * sum + bias for the tile that just finished, then on to the next tile
+        auto finish_tile = [&]() {
+            sts32(wsb_s + lane * 4, __float_as_uint(__fmul_rn(w0, a.out_scale)));
+            sts32(wsb_s + 128 + lane * 4, __float_as_uint(__fmul_rn(w1, a.out_scale)));
+            sts32(wsb_s + 256 + lane * 4, __float_as_uint(b0));
+            sts32(wsb_s + 384 + lane * 4, __float_as_uint(b1));
+            if (tc > 0)   // the strips of the previous tile have been read by every warp
+                ok = mbar_wait_warp(&c->strips_free, (tc - 1) & 1, c, a.status, 9u);
+            __syncwarp();
+            if (!ok) return;
+#pragma unroll
+            for (int j = 0; j < kBN / 2; j += 4) {
+                float o0, o1, o2, o3;
+                unpack2(yacc[j / 2], o0, o1);
+                unpack2(yacc[j / 2 + 1], o2, o3);
+                const uint4 s4 = lds128(wsb_s + j * 4), b4 = lds128(wsb_s + 256 + j * 4);
+                o0 = __fmaf_rn(__uint_as_float(s4.x), o0, __uint_as_float(b4.x));
+                o1 = __fmaf_rn(__uint_as_float(s4.y), o1, __uint_as_float(b4.y));
+                o2 = __fmaf_rn(__uint_as_float(s4.z), o2, __uint_as_float(b4.z));
+                o3 = __fmaf_rn(__uint_as_float(s4.w), o3, __uint_as_float(b4.w));
+                if (YBF16) {
+                    __nv_bfloat162 lo = __floats2bfloat162_rn(o0, o1);
+                    __nv_bfloat162 hi = __floats2bfloat162_rn(o2, o3);
+                    const uint32_t byte = j * 2;   // 8 bytes inside chunk byte / 16
+                    sts64(strip_s + (((byte >> 4) ^ swz) << 4) + (byte & 15), *reinterpret_cast<uint32_t*>(&lo),
+                          *reinterpret_cast<uint32_t*>(&hi));
+                } else {
+                    sts128(strip_s + (((uint32_t)(j >> 2) ^ swz) << 4), __float_as_uint(o0), __float_as_uint(o1),
+                           __float_as_uint(o2), __float_as_uint(o3));
+                }
+            }
+            __syncwarp();
+            mbar_arrive_lane0(&c->strips_ready, lane);
+            ok = mbar_wait_warp(&c->strips_ready, tc & 1, c, a.status, 10u);
+            if (!ok) return;
+            // warp pw writes tile rows 16 pw .. 16 pw + 15 from the strips
+            if (a.vec_ok) {   // one instruction covers 512 contiguous bytes of y
+                constexpr int kRowsPerInstr = YBF16 ? 2 : 1;       // a tile row is 128 * esz bytes
+                const int sub_row = lane / (32 / kRowsPerInstr);
+                const int chunk = lane % (32 / kRowsPerInstr);     // 16-byte chunk of the tile row
+                const int half = chunk / kChunksPerStrip, cs = chunk % kChunksPerStrip;
+                const int64_t col = (int64_t)nt * kBN + chunk * (16 / esz);
+#pragma unroll 4
+                for (int rr = 0; rr < 16; rr += kRowsPerInstr) {
+                    const int r = pw * 16 + rr + sub_row;
+                    const int64_t mg = (int64_t)mt * kBM + r;
+                    const uint32_t src = strips_s + (uint32_t)((half * 4 + (r >> 5)) * 32 + (r & 31)) * kStripBytes +
+                                         (((uint32_t)cs ^ ((uint32_t)r & (kChunksPerStrip - 1))) << 4);
+                    if (mg < a.M && col < a.O) {
+                        const uint4 v = lds128(src);
+                        __stcs(reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(a.y) +
+                                                        ((size_t)mg * a.y_stride + col) * esz), v);
+                    }
+                }
+            } else {          // any alignment: element by element
+#pragma unroll 1
+                for (int rr = 0; rr < 16; ++rr) {
+                    const int r = pw * 16 + rr;
+                    const int64_t mg = (int64_t)mt * kBM + r;
+                    if (mg >= a.M) break;
+#pragma unroll 1
+                    for (int cc = lane; cc < kBN; cc += 32) {
+                        const int64_t col = (int64_t)nt * kBN + cc;
+                        if (col >= a.O) break;
+                        const uint32_t byte = (uint32_t)(cc & 63) * esz;
+                        const uint32_t src = strips_s + (uint32_t)(((cc >> 6) * 4 + (r >> 5)) * 32 + (r & 31)) * kStripBytes +
+                                             (((byte >> 4) ^ ((uint32_t)r & (kChunksPerStrip - 1))) << 4) + (byte & 12u);
+                        const uint32_t word = lds32(src);
+                        if (YBF16)
+                            reinterpret_cast<uint16_t*>(a.y)[mg * a.y_stride + col] =
+                                (uint16_t)((byte & 2) ? (word >> 16) : (word & 0xffffu));
+                        else
+                            reinterpret_cast<uint32_t*>(a.y)[mg * a.y_stride + col] = word;
+                    }
+                }
+            }
+            __syncwarp();
+            mbar_arrive_lane0(&c->strips_free, lane);
+            ++tc;
+            // next tile, next item
+            if (++nt == nt_end) {
+                mbar_arrive_lane0(&c->a_empty, lane);
+                item += gridDim.x;
+                ++ic;
+                if (item < n_items) begin_item();
+            }
+            if (ok && item < n_items) begin_tile();
+        };
+        // One group.  Its first 32 columns were requested earlier and land in va; request the
+        // second 32 into vb and fold va in meanwhile; then release the slot, request the next
+        // group's first half and fold vb in.  The last request is issued even after the last group
+        // (it re-reads an idle slot) so that the landing buffers are written on every path.
+        auto promote = [&]() {
+            const uint32_t dbits = lds32(scale_s);
+            scale_s += kScaleBlock;
+            const uint64_t d2 = pack2(dbits, dbits);
+            tmem_ld_wait();                               // va has landed
+            tmem_ld32(tmem_row + slot * kBN + 32, vb);
+            if (DBG) {
+                if (a.acc_debug && row_ok) debug_store<I8>(a, va, m, n0, a.Kg - grp_left);
+            }
+            if (I8) {
+#pragma unroll
+                for (int q = 0; q < 32; ++q) va[q] = __float_as_uint((float)(int32_t)va[q]);
+            }
+#pragma unroll
+            for (int q = 0; q < 16; ++q) fma2(yacc[q], pack2(va[2 * q], va[2 * q + 1]), d2);
+            tmem_ld_wait();                               // vb has landed: the slot is drained
+            tc_fence_before();
+            __syncwarp();
+            mbar_arrive_lane0(&c->tempty[slot], lane);
+            slot = (slot + 1) & (kSlots - 1);
+            tph ^= (slot == 0);
+            if (++gc < total) ok = mbar_wait_warp(&c->tfull[slot], tph, c, a.status, 2u);
+            tc_fence_after();
+            tmem_ld32(tmem_row + slot * kBN, va);
+            if (DBG) {
+                if (a.acc_debug && row_ok) debug_store<I8>(a, vb, m, n0 + 32, a.Kg - grp_left);
+            }
+            if (I8) {
+#pragma unroll
+                for (int q = 0; q < 32; ++q) vb[q] = __float_as_uint((float)(int32_t)vb[q]);
+            }
+#pragma unroll
+            for (int q = 0; q < 16; ++q) fma2(yacc[16 + q], pack2(vb[2 * q], vb[2 * q + 1]), d2);
+            if (--grp_left == 0 && ok) finish_tile();
+        };
+
+        if (total > 0) {
+            begin_item();
+            if (ok) {
+                begin_tile();
+                ok = mbar_wait_warp(&c->tfull[0], 0, c, a.status, 2u);
+            }
+            tc_fence_after();
+            tmem_ld32(tmem_row, va);
+#pragma unroll 1
+            while (ok && gc < total) promote();
+        }
+        tmem_ld_wait();            // nothing may still be landing when TMEM is released
     }
 
     tc_fence_before();
@@ -360,10 +694,70 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_linear_kernel(LinArgs a) {
     if (warp == kMmaWarp) {
         // all MMAs this CTA issued have completed unless a wait gave up; in that case give the
         // tensor core a moment before the columns are handed back
-        if (sm->abort_flag) __nanosleep(1000000);
+        if (c->abort_flag) __nanosleep(1000000);
         __syncwarp();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
+}
+
+// ------------------------------------------------------------------------------------------
+// host side
+
+struct Plan {
+    int64_t tiles_m, tiles_n;
+    int32_t n_steps, n_chunks, Kg, n_parts, a_resident, n_stages;
+    uint32_t ares_off, ring_off, stage_bytes, staging_off, wsb_off, smem_bytes;
+    size_t a_bytes, b_bytes, s_bytes;   // operand and scale blocks in the workspace
+};
+
+constexpr size_t kWorkspaceHeader = 256;   // status word, then the blocks
+
+// false: sizes out of range, or the problem's scales plus two ring stages do not fit in shared memory
+bool make_plan(int64_t M, int64_t I_pad, int64_t O, int32_t g, int n_sm, Plan& p) {
+    p.tiles_m = (M + kBM - 1) / kBM;
+    p.tiles_n = (O + kBN - 1) / kBN;
+    if (p.tiles_m > INT32_MAX / 4096 || p.tiles_n > INT32_MAX / 4096 || I_pad / 32 > INT32_MAX / 8) return false;
+    p.n_steps = (int32_t)(I_pad / 32);
+    p.n_chunks = (p.n_steps + kChunk - 1) / kChunk;
+    p.Kg = (int32_t)(I_pad / g);
+    p.a_bytes = (size_t)p.tiles_m * p.n_steps * kBlock;
+    p.b_bytes = (size_t)p.tiles_n * p.n_steps * kBlock;
+    p.s_bytes = (size_t)p.tiles_m * p.Kg * kScaleBlock;
+    // shared memory: control, the item's scales, [resident A], ring, output strips, channel scales
+    const int64_t scales = (int64_t)p.Kg * kScaleBlock;
+    const int64_t fixed = 128 + kCtrlBytes + scales + kStagingBytes + kWsbBytes;
+    const int64_t a_res = (int64_t)p.n_steps * kBlock;
+    const int64_t stage_b = (int64_t)kChunk * kBlock, stage_ab = 2 * stage_b;
+    const int64_t stages_res = (kSmemLimit - fixed - a_res) / stage_b;
+    p.ares_off = (uint32_t)(kCtrlBytes + scales);
+    if (stages_res >= 3) {
+        p.a_resident = 1;
+        p.n_stages = (int32_t)(stages_res > kMaxStages ? kMaxStages : stages_res);
+        p.stage_bytes = (uint32_t)stage_b;
+        p.ring_off = p.ares_off + (uint32_t)a_res;
+    } else {
+        const int64_t st = (kSmemLimit - fixed) / stage_ab;
+        if (st < 2) return false;
+        p.a_resident = 0;
+        p.n_stages = (int32_t)(st > kMaxStages ? kMaxStages : st);
+        p.stage_bytes = (uint32_t)stage_ab;
+        p.ring_off = p.ares_off;
+    }
+    p.staging_off = p.ring_off + (uint32_t)p.n_stages * p.stage_bytes;
+    p.wsb_off = p.staging_off + kStagingBytes;
+    p.smem_bytes = p.wsb_off + kWsbBytes + 128;
+    // split the column tiles of a row block into parts so that the items fill the SMs evenly
+    int best = 1;
+    int64_t best_cost = INT64_MAX;
+    for (int parts = 1; parts <= p.tiles_n; ++parts) {
+        const int64_t items = p.tiles_m * parts;
+        const int64_t waves = (items + n_sm - 1) / n_sm;
+        const int64_t per_item = (p.tiles_n + parts - 1) / parts;
+        const int64_t cost = waves * (per_item * 16 + 1);   // +1: an item reloads its A block
+        if (cost < best_cost) { best_cost = cost; best = parts; }
+    }
+    p.n_parts = best;
+    return true;
 }
 
 }  // namespace
@@ -371,7 +765,23 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_linear_kernel(LinArgs a) {
 
 using namespace tdq;
 
-extern "C" size_t tdq_linear_workspace_bytes(int64_t, int64_t, int64_t, int32_t) { return 256; }
+static int sm_count() {
+    static int n_sm = 0;
+    if (n_sm == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+        if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n_sm = 0;
+    }
+    return n_sm;
+}
+
+extern "C" size_t tdq_linear_workspace_bytes(int64_t M, int64_t I_pad, int64_t O, int32_t group_size) {
+    if (M < 0 || I_pad <= 0 || O <= 0 || group_size <= 0 || group_size % 32 || I_pad % group_size)
+        return kWorkspaceHeader;
+    Plan p;
+    if (!make_plan(M, I_pad, O, group_size, 148, p)) return kWorkspaceHeader;
+    return kWorkspaceHeader + p.a_bytes + p.b_bytes + p.s_bytes;
+}
 
 extern "C" tdq_status tdq_w4a4_linear(const uint8_t* xcodes, const float* xscale, const uint8_t* wcodes,
                                       const float* wscale, const float* bias, int64_t M, int64_t I_pad, int64_t O,
@@ -383,55 +793,71 @@ extern "C" tdq_status tdq_w4a4_linear(const uint8_t* xcodes, const float* xscale
     if (y_dtype != TDQ_F32 && y_dtype != TDQ_BF16) return TDQ_ERR_INVALID_ARG;
     if (group_size <= 0 || I_pad % group_size) return TDQ_ERR_INVALID_ARG;
     if (group_size % 32 || group_size > 4096) return TDQ_ERR_UNSUPPORTED;
-    if (!workspace || workspace_bytes < tdq_linear_workspace_bytes(M, I_pad, O, group_size)) return TDQ_ERR_WORKSPACE;
+    if (I_pad / 2 > INT32_MAX) return TDQ_ERR_INVALID_ARG;
+    Plan p;
+    if (!make_plan(M, I_pad, O, group_size, 148, p)) return TDQ_ERR_UNSUPPORTED;
+    if (!workspace || workspace_bytes < kWorkspaceHeader + p.a_bytes + p.b_bytes + p.s_bytes) return TDQ_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(xcodes) % 16 || reinterpret_cast<uintptr_t>(wcodes) % 16 ||
         reinterpret_cast<uintptr_t>(workspace) % 16)
         return TDQ_ERR_ALIGNMENT;
-    if (I_pad / 2 > INT32_MAX) return TDQ_ERR_INVALID_ARG;
     if (M == 0) return TDQ_OK;
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    const int n_sm = sm_count();
+    if (n_sm <= 0) return TDQ_ERR_CUDA;
+    if (!make_plan(M, I_pad, O, group_size, n_sm, p)) return TDQ_ERR_UNSUPPORTED;
+
+    uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+    const bool i8 = group_size > 32;   // several instructions chain into one slot: keep the integer accumulator
+
+    ExpandArgs e;
+    e.xcodes = xcodes; e.xscale = xscale; e.wcodes = wcodes;
+    e.a_blocks = ws + kWorkspaceHeader;
+    e.b_blocks = e.a_blocks + p.a_bytes;
+    e.s_blocks = e.b_blocks + p.b_bytes;
+    e.M = M; e.O = O;
+    e.row_bytes = (int32_t)(I_pad / 2);
+    e.n_steps = p.n_steps; e.n_chunks = p.n_chunks;
+    e.steps_per_grp = group_size / 32;
+    e.Kg = p.Kg;
+    e.tiles_m = (int32_t)p.tiles_m; e.tiles_n = (int32_t)p.tiles_n;
 
     LinArgs a;
-    a.xcodes = xcodes; a.xscale = xscale; a.wcodes = wcodes; a.wscale = wscale; a.bias = bias;
+    a.a_blocks = e.a_blocks; a.b_blocks = e.b_blocks; a.s_blocks = e.s_blocks;
+    a.wscale = wscale; a.bias = bias;
     a.M = M; a.O = O;
-    a.row_bytes = (int32_t)(I_pad / 2);
-    a.n_steps = (int32_t)(I_pad / 32);
-    a.steps_per_grp = group_size / 32;
-    a.Kg = (int32_t)(I_pad / group_size);
-    const int64_t tm = (M + kBM - 1) / kBM, tn = (O + kBN - 1) / kBN;
-    if (tm > INT32_MAX || tn > INT32_MAX) return TDQ_ERR_INVALID_ARG;
-    a.tiles_m = (int32_t)tm;
-    a.tiles_n = (int32_t)tn;
+    a.n_steps = p.n_steps; a.steps_per_grp = e.steps_per_grp; a.Kg = p.Kg;
+    a.tiles_m = e.tiles_m; a.tiles_n = e.tiles_n; a.n_parts = p.n_parts;
+    a.a_resident = p.a_resident; a.n_stages = p.n_stages;
+    a.ares_off = p.ares_off; a.ring_off = p.ring_off; a.stage_bytes = p.stage_bytes;
+    a.staging_off = p.staging_off; a.wsb_off = p.wsb_off;
     a.y = y; a.y_stride = y_row_stride; a.acc_debug = acc_debug;
     a.status = reinterpret_cast<uint32_t*>(workspace);
-    a.vec_ok = (reinterpret_cast<uintptr_t>(y) % 16 == 0 && reinterpret_cast<uintptr_t>(wscale) % 16 == 0 &&
-                (!bias || reinterpret_cast<uintptr_t>(bias) % 16 == 0) && y_row_stride % 4 == 0)
-                   ? 1
-                   : 0;
+    const int64_t esz = y_dtype == TDQ_BF16 ? 2 : 4;
+    // vector stores: every 16-byte chunk of a tile row is aligned and lies wholly inside or outside y
+    a.vec_ok = (reinterpret_cast<uintptr_t>(y) % 16 == 0 && (y_row_stride * esz) % 16 == 0 && (O * esz) % 16 == 0) ? 1 : 0;
+    a.out_scale = i8 ? 0.00390625f : 262144.0f;
 
-    static int n_sm = 0;
-    if (n_sm == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return TDQ_ERR_CUDA;
-        if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return TDQ_ERR_CUDA;
-    }
-    const size_t smem = sizeof(Smem) + 128;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(w4a4_linear_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-                cudaSuccess ||
-            cudaFuncSetAttribute(w4a4_linear_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-                cudaSuccess)
-            return TDQ_ERR_CUDA;
-        attr_set = true;
-    }
+    const bool ybf = y_dtype == TDQ_BF16, dbg = acc_debug != nullptr;
+    void (*kernel)(LinArgs) = nullptr;
+#define TDQ_PICK(I8_, YB_, DBG_) if (i8 == I8_ && ybf == YB_ && dbg == DBG_) kernel = w4a4_gemm_kernel<I8_, YB_, DBG_>;
+    TDQ_PICK(false, false, false) TDQ_PICK(false, true, false) TDQ_PICK(true, false, false) TDQ_PICK(true, true, false)
+    TDQ_PICK(false, false, true) TDQ_PICK(false, true, true) TDQ_PICK(true, false, true) TDQ_PICK(true, true, true)
+#undef TDQ_PICK
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess)
+        return TDQ_ERR_CUDA;
     if (cudaMemsetAsync(workspace, 0, 16, stream) != cudaSuccess) return TDQ_ERR_CUDA;
-    const int64_t tiles = tm * tn;
-    const unsigned grid = (unsigned)(tiles < n_sm ? tiles : n_sm);
-    if (y_dtype == TDQ_BF16)
-        w4a4_linear_kernel<true><<<grid, kThreads, smem, stream>>>(a);
+
+    const unsigned pieces = (unsigned)((p.tiles_m + p.tiles_n) * p.n_chunks);
+    if (i8)
+        expand_kernel<true><<<pieces, kExpandThreads, 0, stream>>>(e);
     else
-        w4a4_linear_kernel<false><<<grid, kThreads, smem, stream>>>(a);
+        expand_kernel<false><<<pieces, kExpandThreads, 0, stream>>>(e);
+    if (cudaGetLastError() != cudaSuccess) return TDQ_ERR_CUDA;
+    g_launch_count.fetch_add(1, std::memory_order_relaxed);
+
+    const int64_t items = p.tiles_m * p.n_parts;
+    const unsigned grid = (unsigned)(items < n_sm ? items : n_sm);
+    kernel<<<grid, kThreads, p.smem_bytes, stream>>>(a);
     if (cudaGetLastError() != cudaSuccess) return TDQ_ERR_CUDA;
     g_launch_count.fetch_add(1, std::memory_order_relaxed);
     return TDQ_OK;

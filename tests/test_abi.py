@@ -63,7 +63,7 @@ def test_bad_arguments_return_codes_without_launching(tdq):
     assert L.tdq_quantize_weight(None, 0, 4, 64, 32, fake, fake, None) == tdq.ERR_INVALID_ARG
     assert L.tdq_quantize_weight(fake, 0, 4, 64, 3, fake, fake, None) == tdq.ERR_INVALID_ARG
     assert L.tdq_quantize_weight(fake, 0, 0, 64, 32, fake, fake, None) == tdq.OK
-    ws = 256
+    ws = 1 << 20
     lin = lambda *a: L.tdq_w4a4_linear(*a)
     assert lin(None, fake, fake, fake, None, 4, 64, 8, 32, fake, 0, 8, None, fake, ws, None) == tdq.ERR_INVALID_ARG
     assert lin(fake, fake, fake, fake, None, 4, 64, 8, 48, fake, 0, 8, None, fake, ws, None) == tdq.ERR_INVALID_ARG
