@@ -140,6 +140,35 @@ tdq_status tdq_quant_linear_host(const void* x_host /* HOST */, tdq_dtype x_dtyp
                                  void* x_dev, uint8_t* codes_dev, float* scale_dev, void* y_dev,
                                  void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/*
+ * tdq_w4a4_linear for callers that cannot allocate device memory.  (An addition of this library:
+ * the paper has no counterpart.)  Some code that wants to run the linear layer has no way to
+ * obtain a workspace: a plug-in running inside a host application that owns all device memory,
+ * a callback where calling cudaMalloc is forbidden or would synchronise the whole device, a
+ * process whose memory budget was handed out up front.  This entry point computes exactly what
+ * tdq_w4a4_linear computes, with the same argument meaning and checks, but keeps the operand
+ * blocks and the status word in an array that is part of the library image itself
+ * (TDQ_LINEAR_STATIC_BYTES, 8 MiB, in every CUDA context that loads the library,
+ * from load until the process exits).  It calls no allocating or freeing routine.
+ *   - Problems whose tdq_linear_workspace_bytes() exceed the capacity are refused with
+ *     TDQ_ERR_WORKSPACE and nothing is launched (of the five benchmark workloads the first
+ *     three fit).  There is no acc_debug output.
+ *   - The first call on each device, made with that device current, looks up where the array
+ *     lives on that device; make that first call outside any stream capture.
+ *   - All calls share the one array, which keeps whatever the last call left in it.  Every call
+ *     rewrites all the blocks it is going to read and clears the status word, so earlier
+ *     contents never leak into a result; but two calls that overlap on the GPU (different
+ *     streams, or different host threads) race on it.  Order them on one stream.
+ *   - wait != 0: the call returns only after its work on cuda_stream has finished, and answers
+ *     TDQ_ERR_DEVICE_TIMEOUT if a bounded wait inside the kernel ran out.  wait == 0: the call
+ *     is asynchronous like tdq_w4a4_linear and that condition goes unreported.
+ */
+#define TDQ_LINEAR_STATIC_BYTES ((size_t)8 << 20)
+tdq_status tdq_w4a4_linear_static(const uint8_t* xcodes, const float* xscale, const uint8_t* wcodes,
+                                  const float* wscale, const float* bias, int64_t M, int64_t I_pad, int64_t O,
+                                  int32_t group_size, void* y, tdq_dtype y_dtype, int64_t y_row_stride,
+                                  int32_t wait, void* cuda_stream);
+
 /* Bytes of workspace tdq_w4a4_linear / tdq_quant_linear_fused need for this problem. */
 size_t tdq_linear_workspace_bytes(int64_t M, int64_t I_pad, int64_t O, int32_t group_size);
 

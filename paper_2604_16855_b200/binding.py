@@ -23,7 +23,7 @@ ENABLE_C1, ENABLE_C2 = 1, 2
 # every symbol include/tdq.h declares
 EXPORTS = ["tdq_default_act_params", "tdq_quantize_act", "tdq_quantize_weight", "tdq_w4a4_linear",
            "tdq_quant_linear_fused", "tdq_quant_linear_host", "tdq_linear_workspace_bytes",
-           "tdq_workspace_status", "tdq_status_string", "tdq_kernel_launch_count"]
+           "tdq_workspace_status", "tdq_status_string", "tdq_kernel_launch_count", "tdq_w4a4_linear_static"]
 
 
 class ActParams(ctypes.Structure):
@@ -42,6 +42,9 @@ _lib.tdq_quantize_weight.restype = ctypes.c_int
 _lib.tdq_w4a4_linear.argtypes = [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp, ctypes.c_int, _i64,
                                  _vp, _vp, _sz, _vp]
 _lib.tdq_w4a4_linear.restype = ctypes.c_int
+_lib.tdq_w4a4_linear_static.argtypes = [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp, ctypes.c_int, _i64,
+                                        _i32, _vp]
+_lib.tdq_w4a4_linear_static.restype = ctypes.c_int
 _lib.tdq_quant_linear_fused.argtypes = [_vp, ctypes.c_int, _i64, _i64, _i64, _i64, _pp, _vp, _vp, _vp, _i64,
                                         _vp, ctypes.c_int, _i64, _vp, _sz, _vp]
 _lib.tdq_quant_linear_fused.restype = ctypes.c_int
@@ -173,6 +176,23 @@ def w4a4_linear(xcodes, xscale, wcodes, wscale, bias=None, *, g=32, out_dtype=to
     _check(_lib.tdq_w4a4_linear(_ptr(xcodes), _ptr(xscale), _ptr(wcodes), _ptr(wscale), _ptr(bias), M, I_pad, O, g,
                                 _ptr(y), _dtype_id(y), y.stride(0) if M > 0 else O, _ptr(acc_debug),
                                 _ptr(workspace), workspace.numel(), _stream(xcodes)), "tdq_w4a4_linear")
+    return y
+
+
+LINEAR_STATIC_BYTES = 8 << 20   # TDQ_LINEAR_STATIC_BYTES of the header
+
+
+def w4a4_linear_static(xcodes, xscale, wcodes, wscale, bias=None, *, g=32, y, wait=True):
+    """tdq_w4a4_linear_static: the linear layer for callers that may not allocate device memory.
+
+    The scratch space is a fixed array inside the library, so this wrapper allocates nothing
+    either: the caller passes the output tensor y [M, O].  Returns y."""
+    _need_cuda(xcodes, xscale, wcodes, wscale, bias, y)
+    M, half = xcodes.shape
+    O = wcodes.shape[0]
+    _check(_lib.tdq_w4a4_linear_static(_ptr(xcodes), _ptr(xscale), _ptr(wcodes), _ptr(wscale), _ptr(bias), M, half * 2,
+                                       O, g, _ptr(y), _dtype_id(y), y.stride(0) if M > 0 else O, 1 if wait else 0,
+                                       _stream(xcodes)), "tdq_w4a4_linear_static")
     return y
 
 

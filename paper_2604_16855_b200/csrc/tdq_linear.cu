@@ -48,6 +48,8 @@
 // Every wait on an mbarrier is bounded: after about a second the thread records a code in the
 // workspace status word and raises a CTA-wide flag; every role then leaves its loops, the CTA
 // releases its TMEM and returns.
+#include <mutex>
+
 #include "tdq_common.cuh"
 
 namespace tdq {
@@ -871,4 +873,49 @@ extern "C" tdq_status tdq_workspace_status(const void* workspace, void* cuda_str
     if (cudaStreamSynchronize(stream) != cudaSuccess) return TDQ_ERR_CUDA;
     if (detail) *detail = word;
     return word == 0 ? TDQ_OK : TDQ_ERR_DEVICE_TIMEOUT;
+}
+
+// ------------------------------------------------------------------------------------------
+// tdq_w4a4_linear_static: the same two kernels, with the operand blocks in a fixed device array
+
+namespace {
+constexpr size_t kStaticScratchBytes = TDQ_LINEAR_STATIC_BYTES;
+// Lives in every CUDA context that loads this library, from load to exit.  Host code may only
+// use the name to look its device address up; the kernels get that address as a plain pointer.
+static __device__ __align__(256) uint8_t g_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_ptr[kMaxDevices] = {};
+}  // namespace
+
+extern "C" tdq_status tdq_w4a4_linear_static(const uint8_t* xcodes, const float* xscale, const uint8_t* wcodes,
+                                             const float* wscale, const float* bias, int64_t M, int64_t I_pad,
+                                             int64_t O, int32_t group_size, void* y, tdq_dtype y_dtype,
+                                             int64_t y_row_stride, int32_t wait, void* cuda_stream) {
+    // the argument checks that do not depend on the scratch come first, as in tdq_w4a4_linear
+    if (!xcodes || !xscale || !wcodes || !wscale || !y) return TDQ_ERR_INVALID_ARG;
+    if (M < 0 || O <= 0 || I_pad <= 0 || y_row_stride < O) return TDQ_ERR_INVALID_ARG;
+    if (group_size <= 0 || I_pad % group_size) return TDQ_ERR_INVALID_ARG;
+    if (group_size % 32 || group_size > 4096) return TDQ_ERR_UNSUPPORTED;
+    const size_t need = tdq_linear_workspace_bytes(M, I_pad, O, group_size);
+    if (need > kStaticScratchBytes) return TDQ_ERR_WORKSPACE;   // the problem is too large for the fixed array
+
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return TDQ_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return TDQ_ERR_UNSUPPORTED;
+    void* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!g_static_ptr[dev]) {   // first call on this device: ask the runtime where the array lives here
+            void* p = nullptr;
+            if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return TDQ_ERR_CUDA;
+            g_static_ptr[dev] = p;
+        }
+        scratch = g_static_ptr[dev];
+    }
+    tdq_status st = tdq_w4a4_linear(xcodes, xscale, wcodes, wscale, bias, M, I_pad, O, group_size, y, y_dtype,
+                                    y_row_stride, nullptr, scratch, kStaticScratchBytes, cuda_stream);
+    if (st != TDQ_OK || !wait || M == 0) return st;
+    return tdq_workspace_status(scratch, cuda_stream, nullptr);
 }
