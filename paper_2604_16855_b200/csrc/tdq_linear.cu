@@ -630,6 +630,10 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
             ++tc;
             // next tile, next item
             if (++nt == nt_end) {
+                // the item's scales were read through the generic proxy; the next item's bulk copies
+                // overwrite them through the async proxy, which only a proxy fence orders after the reads
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
                 mbar_arrive_lane0(&c->a_empty, lane);
                 item += gridDim.x;
                 ++ic;

@@ -169,55 +169,10 @@ __device__ __forceinline__ uint32_t nibble_ieee(float x, float c, float delta) {
     return (uint32_t)quantize_ieee(x, c, delta) & 0xFu;
 }
 
+// One group held in registers (w: 16 packed bf16 pairs or 32 floats, in channel order): statistics,
+// projection, quantization; writes the group's 16 code bytes and its scale.
 template <bool BF16, int KZR>
-__global__ void __launch_bounds__(kFastThreads) act_g32_kernel(ActArgs a) {
-    constexpr int kGroupBytes = BF16 ? 64 : 128;
-    constexpr int kChunks = kGroupBytes / 16;          // 16-byte chunks per group
-    constexpr int kSwzMask = kChunks - 1;
-    __shared__ __align__(16) uint4 tile[kFastThreads * kChunks];
-
-    const int t = threadIdx.x;
-    const int64_t g0 = (int64_t)blockIdx.x * kFastThreads;
-    const char* xb = reinterpret_cast<const char*>(a.x);
-    const int64_t esize = BF16 ? 2 : 4;
-    const bool flat = (a.row_stride == a.C);
-
-    // stage: coalesced 16-byte loads; chunk p of local group l lands at l*kChunks + (p ^ swz(l))
-#pragma unroll
-    for (int j = 0; j < kChunks; ++j) {
-        const int ch = t + j * kFastThreads;
-        const int l = ch / kChunks, p = ch % kChunks;
-        const int64_t gi = g0 + l;
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (gi < a.total_groups) {
-            int64_t off;
-            if (flat) {
-                off = gi * kGroupBytes + p * 16;
-            } else {
-                const int64_t m = gi / a.K;
-                const int64_t k = gi - m * a.K;
-                off = (m * a.row_stride + k * 32) * esize + p * 16;
-            }
-            v = __ldg(reinterpret_cast<const uint4*>(xb + off));
-        }
-        const int swz = BF16 ? ((l >> 1) & kSwzMask) : (l & kSwzMask);
-        tile[l * kChunks + (p ^ swz)] = v;
-    }
-    __syncthreads();
-
-    const int64_t gi = g0 + t;
-    if (gi >= a.total_groups) return;
-
-    // this thread's group: words w[], 16 packed bf16 pairs or 32 floats
-    uint32_t w[kChunks * 4];
-    {
-        const int swz = BF16 ? ((t >> 1) & kSwzMask) : (t & kSwzMask);
-#pragma unroll
-        for (int p = 0; p < kChunks; ++p) {
-            uint4 v = tile[t * kChunks + (p ^ swz)];
-            w[4 * p + 0] = v.x; w[4 * p + 1] = v.y; w[4 * p + 2] = v.z; w[4 * p + 3] = v.w;
-        }
-    }
+__device__ __forceinline__ void process_group(const uint32_t (&w)[BF16 ? 16 : 32], const ActArgs& a, int64_t gi) {
     auto get = [&](int i) -> float {
         if (BF16) return (i & 1) ? __uint_as_float(w[i >> 1] & 0xffff0000u) : __uint_as_float(w[i >> 1] << 16);
         return __uint_as_float(w[i]);
@@ -319,10 +274,197 @@ __global__ void __launch_bounds__(kFastThreads) act_g32_kernel(ActArgs a) {
     if (a.offset) a.offset[gi] = 0.0f;
 }
 
+template <bool BF16, int KZR>
+__global__ void __launch_bounds__(kFastThreads) act_g32_kernel(ActArgs a) {
+    constexpr int kGroupBytes = BF16 ? 64 : 128;
+    constexpr int kChunks = kGroupBytes / 16;          // 16-byte chunks per group
+    constexpr int kSwzMask = kChunks - 1;
+    __shared__ __align__(16) uint4 tile[kFastThreads * kChunks];
+
+    const int t = threadIdx.x;
+    const int64_t g0 = (int64_t)blockIdx.x * kFastThreads;
+    const char* xb = reinterpret_cast<const char*>(a.x);
+    const int64_t esize = BF16 ? 2 : 4;
+    const bool flat = (a.row_stride == a.C);
+
+    // stage: coalesced 16-byte loads; chunk p of local group l lands at l*kChunks + (p ^ swz(l))
+#pragma unroll
+    for (int j = 0; j < kChunks; ++j) {
+        const int ch = t + j * kFastThreads;
+        const int l = ch / kChunks, p = ch % kChunks;
+        const int64_t gi = g0 + l;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (gi < a.total_groups) {
+            int64_t off;
+            if (flat) {
+                off = gi * kGroupBytes + p * 16;
+            } else {
+                const int64_t m = gi / a.K;
+                const int64_t k = gi - m * a.K;
+                off = (m * a.row_stride + k * 32) * esize + p * 16;
+            }
+            v = __ldg(reinterpret_cast<const uint4*>(xb + off));
+        }
+        const int swz = BF16 ? ((l >> 1) & kSwzMask) : (l & kSwzMask);
+        tile[l * kChunks + (p ^ swz)] = v;
+    }
+    __syncthreads();
+
+    const int64_t gi = g0 + t;
+    if (gi >= a.total_groups) return;
+
+    // this thread's group: words w[], 16 packed bf16 pairs or 32 floats
+    uint32_t w[kChunks * 4];
+    {
+        const int swz = BF16 ? ((t >> 1) & kSwzMask) : (t & kSwzMask);
+#pragma unroll
+        for (int p = 0; p < kChunks; ++p) {
+            uint4 v = tile[t * kChunks + (p ^ swz)];
+            w[4 * p + 0] = v.x; w[4 * p + 1] = v.y; w[4 * p + 2] = v.z; w[4 * p + 3] = v.w;
+        }
+    }
+    process_group<BF16, KZR>(w, a, gi);
+}
+
+// ------------------------------------------------------------------------------------------
+// fast kernel for dense rows (row stride == C): persistent CTAs, bulk-copy ring
+//
+// Consecutive groups are consecutive in memory, so a tile of 256 groups is one contiguous
+// piece (16 KB of bf16, 32 KB of fp32).  A producer lane streams tiles into a ring of
+// shared-memory stages with cp.async.bulk; the 256 consumer threads take one group each out of
+// a stage, hand the stage back, and then spend their time on the selection network while the
+// next tiles are already landing.  Waits are bounded (see kRingTimeout).
+
+constexpr int kRingStagesBf16 = 4, kRingStagesF32 = 3;
+constexpr int kRingThreads = kFastThreads + 32;
+constexpr long long kRingTimeout = 2000000000LL;
+
+__device__ __forceinline__ uint32_t ring_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ bool ring_test(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(ring_smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// false when the phase did not complete in about a second (the caller then stops working)
+__device__ __forceinline__ bool ring_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    if (ring_test(bar, parity)) return true;
+    long long t0 = 0;
+    uint32_t polls = 0;
+#pragma unroll 1
+    while (!ring_test(bar, parity)) {
+        if ((++polls & 63u) == 0u) {
+            if (*abort_flag) return false;
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            if (now - t0 > kRingTimeout) { *abort_flag = 1; return false; }
+        }
+    }
+    return true;
+}
+
+template <bool BF16, int KZR>
+__global__ void __launch_bounds__(kRingThreads) act_g32_ring_kernel(ActArgs a, int64_t n_tiles) {
+    constexpr int kGroupBytes = BF16 ? 64 : 128;
+    constexpr int kChunks = kGroupBytes / 16;
+    constexpr int kStages = BF16 ? kRingStagesBf16 : kRingStagesF32;
+    constexpr int kStageBytes = kFastThreads * kGroupBytes;
+    extern __shared__ __align__(128) uint8_t ring_smem[];
+    __shared__ uint64_t full[kStages], empty[kStages];
+    __shared__ volatile int abort_flag;
+    const int t = threadIdx.x;
+    if (t == 0) {
+        for (int i = 0; i < kStages; ++i) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(ring_smem_u32(&full[i])), "r"(1) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(ring_smem_u32(&empty[i])), "r"(kFastThreads / 32) : "memory");
+        }
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const char* xb = reinterpret_cast<const char*>(a.x);
+    if (t >= kFastThreads) {
+        if (t == kFastThreads) {   // producer lane
+            uint32_t s = 0, ph = 0;
+            for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+                if (!ring_wait(&empty[s], ph ^ 1, &abort_flag)) break;
+                const int64_t g0 = tile * kFastThreads;
+                const int64_t ng = min((int64_t)kFastThreads, a.total_groups - g0);
+                const uint32_t bytes = (uint32_t)(ng * kGroupBytes);
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(ring_smem_u32(&full[s])), "r"(bytes) : "memory");
+                asm volatile("cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                             ::"r"(ring_smem_u32(ring_smem + (size_t)s * kStageBytes)), "l"(xb + g0 * kGroupBytes), "r"(bytes),
+                               "r"(ring_smem_u32(&full[s]))
+                             : "memory");
+                if (++s == kStages) { s = 0; ph ^= 1; }
+            }
+        }
+        return;
+    }
+    uint32_t s = 0, ph = 0;
+    for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+        if (!__all_sync(0xffffffffu, ring_wait(&full[s], ph, &abort_flag))) break;
+        const int64_t gi = tile * kFastThreads + t;
+        uint32_t w[kChunks * 4];
+        // volatile loads: the stage is handed back right below, so these must be the only reads of it
+        const uint32_t src = ring_smem_u32(ring_smem + (size_t)s * kStageBytes + (size_t)t * kGroupBytes);
+#pragma unroll
+        for (int p = 0; p < kChunks; ++p)
+            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(w[4 * p + 0]), "=r"(w[4 * p + 1]), "=r"(w[4 * p + 2]), "=r"(w[4 * p + 3])
+                         : "r"(src + p * 16)
+                         : "memory");
+        // The producer refills the stage through the async proxy as soon as the eighth warp has
+        // arrived.  Reads made through the generic proxy are only ordered before such writes by a
+        // proxy fence; without it the refill was observed to overtake these loads.
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if ((t & 31) == 0)
+            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(ring_smem_u32(&empty[s])) : "memory");
+        if (++s == kStages) { s = 0; ph ^= 1; }
+        if (gi < a.total_groups) process_group<BF16, KZR>(w, a, gi);
+    }
+}
+
+template <bool BF16, int KZR>
+cudaError_t launch_ring(const ActArgs& a, cudaStream_t st) {
+    constexpr int kStages = BF16 ? kRingStagesBf16 : kRingStagesF32;
+    constexpr int smem = kStages * kFastThreads * (BF16 ? 64 : 128);
+    static int n_sm = 0;
+    static bool attr_done = false;
+    if (n_sm == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorUnknown;
+        if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return cudaErrorUnknown;
+    }
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(act_g32_ring_kernel<BF16, KZR>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    const int64_t n_tiles = (a.total_groups + kFastThreads - 1) / kFastThreads;
+    const int64_t grid = n_tiles < 2 * n_sm ? n_tiles : 2 * n_sm;
+    act_g32_ring_kernel<BF16, KZR><<<(unsigned)grid, kRingThreads, smem, st>>>(a, n_tiles);
+    return cudaGetLastError();
+}
+
 template <bool BF16>
 cudaError_t launch_fast(const ActArgs& a, cudaStream_t st) {
     const int64_t blocks = (a.total_groups + kFastThreads - 1) / kFastThreads;
     dim3 grid((unsigned)blocks), block(kFastThreads);
+    if (a.row_stride == a.C) {   // dense rows: the persistent ring kernel
+        switch (a.k_zr) {
+#define TDQ_CASE(KZ) case KZ: return launch_ring<BF16, KZ>(a, st);
+            TDQ_CASE(4) TDQ_CASE(7) TDQ_CASE(10) TDQ_CASE(13) TDQ_CASE(16) TDQ_CASE(32)
+#undef TDQ_CASE
+            default: return cudaErrorInvalidValue;
+        }
+    }
     switch (a.k_zr) {
 #define TDQ_CASE(KZ) case KZ: act_g32_kernel<BF16, KZ><<<grid, block, 0, st>>>(a); break;
         TDQ_CASE(4) TDQ_CASE(7) TDQ_CASE(10) TDQ_CASE(13) TDQ_CASE(16) TDQ_CASE(32)
