@@ -154,13 +154,28 @@ def run_reference(args):
     sample = "first %d of %d token rows of %s per step, quantizer + linear" % (rows, case.M, case.name)
     out = dict(metric=METRIC, impl="reference", value=value, unit="GB/s", n_gpus=args.gpus, steps=args.steps,
                warmup=args.warmup, ms_per_step=1e3 * wall / args.steps, higher_is_better=True, scaling="weak",
-               vs_baseline=None, dtype="f32 quantizer / int32 contraction / f64 scaling", data="synthetic",
+               vs_baseline=None, dtype="f32", data="synthetic",
                config=dict(workload=case.name, x=[int(v) for v in case.x.shape], w=[int(v) for v in case.w.shape],
                            g=32, tau=1.0, zr=0.2, sample=sample),
                kernels=dict(linear=dict(tops=2.0 * args.steps * rows * case.C * case.O / ls / 1e12)),
                cpu_baseline=dict(value=value, unit="GB/s", cores=legs[0]["cores"], kind="oracle", sample=sample),
                e2e=dict(value=value, unit="GB/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
     print(json.dumps(out))
+
+
+def max_over_ranks(values, device, world):
+    """Element-wise maximum of a list of floats over all ranks (the slowest rank sets the time)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.tolist()]
+
+
+def whole_job_rate(units_per_rank, world, ms):
+    """Units all ranks processed per second, given the slowest rank's time in milliseconds."""
+    return world * units_per_rank / (ms * 1e-3)
 
 
 def run_tdq(args):
@@ -264,10 +279,7 @@ def run_tdq(args):
     barrier()
     e2e_ms = e0.elapsed_time(e1)
 
-    times = torch.tensor([total_ms, q_ms, l_ms, e2e_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    total_ms, q_ms, l_ms, e2e_ms = [float(v) for v in times.tolist()]
+    total_ms, q_ms, l_ms, e2e_ms = max_over_ranks([total_ms, q_ms, l_ms, e2e_ms], dev, world)
 
     if rank == 0:
         peaks = load_peaks()
@@ -298,7 +310,7 @@ def run_tdq(args):
         e2e_value = world * qb * e2e_steps / (e2e_ms * 1e-3) / 1e9
         out = dict(metric=METRIC, value=world * q_gbs, unit="GB/s", n_gpus=world, steps=K, warmup=args.warmup,
                    ms_per_step=total_ms / K, higher_is_better=True, scaling="weak", vs_baseline=None,
-                   dtype="f32 quantizer arithmetic on bf16 input / int8 x int8 -> int32 tensor-core contraction / f32 scaling",
+                   dtype="f32",
                    data="synthetic",
                    config=dict(workload=case.name, x=[int(v) for v in case.x.shape], w=[int(v) for v in case.w.shape],
                                g=32, tau=1.0, zr=0.2, y_dtype="f32",

@@ -456,6 +456,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
         } else if (warp == kMmaWarp && lane == 0) {
             // ------------------------------------------------------------ MMA issue (one lane)
             uint32_t s = 0, ph = 0, slot = 0, tph = 0, ic = 0;
+            bool slot_ready = false;   // the early answer about the current slot, if it was yes
             const uint64_t ares_desc = smem_desc(ares_s);
             bool ok = true;
             for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++ic) {
@@ -470,19 +471,26 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
                             if (!ok) break;
                             bdesc = smem_desc(ring_s + s * a.stage_bytes);
                         }
-                        if (sub == 0) {
+                        if (sub == 0 && !slot_ready) {
                             ok = mbar_wait(&c->tempty[slot], tph ^ 1, c, a.status, 3u);
                             if (!ok) break;
                         }
+                        // ask about the next group's slot now: the answer travels while this step is issued
+                        const bool last_sub = sub + 1 == spg;
+                        const uint32_t nslot = (slot + 1) & (kSlots - 1), ntph = tph ^ (nslot == 0);
+                        if (last_sub) slot_ready = mbar_test(&c->tempty[nslot], ntph ^ 1);
                         tc_fence_after();
                         const uint64_t adesc = resident ? ares_desc + (uint64_t)(ks * (kBlock >> 4))
                                                         : bdesc + (uint64_t)((kChunk + kj) * (kBlock >> 4));
                         mma_issue<I8>(tmem_base + slot * kBN, adesc, bdesc + (uint64_t)(kj * (kBlock >> 4)),
                                       sub == 0 ? 0u : 1u);
-                        if (++sub == spg) {
+                        if (last_sub) {
                             sub = 0;
                             mma_commit(&c->tfull[slot]);
-                            if (++slot == kSlots) { slot = 0; tph ^= 1; }
+                            slot = nslot;
+                            tph = ntph;
+                        } else {
+                            ++sub;
                         }
                         if (++kj == kChunk || ks == a.n_steps - 1) {
                             kj = 0;
@@ -651,6 +659,10 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
             const uint64_t d2 = pack2(dbits, dbits);
             tmem_ld_wait();                               // va has landed
             tmem_ld32(tmem_row + slot * kBN + 32, vb);
+            // ask about the next group's slot now; the answer is needed only after the FMAs below
+            const uint32_t nslot = (slot + 1) & (kSlots - 1), ntph = tph ^ (nslot == 0);
+            const bool more = gc + 1 < total;
+            const bool next_ready = more ? mbar_test(&c->tfull[nslot], ntph) : true;
             if (DBG) {
                 if (a.acc_debug && row_ok) debug_store<I8>(a, va, m, n0, a.Kg - grp_left);
             }
@@ -664,11 +676,18 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
             tc_fence_before();
             __syncwarp();
             mbar_arrive_lane0(&c->tempty[slot], lane);
-            slot = (slot + 1) & (kSlots - 1);
-            tph ^= (slot == 0);
-            if (++gc < total) ok = mbar_wait_warp(&c->tfull[slot], tph, c, a.status, 2u);
-            tc_fence_after();
-            tmem_ld32(tmem_row + slot * kBN, va);
+            slot = nslot;
+            tph = ntph;
+            ++gc;
+            // Request the next group's first half before folding vb in, except at the end of a tile:
+            // there the epilogue goes first, because the next group may belong to the next work item,
+            // which cannot start before this warp has handed the current item's buffers back.
+            const bool tile_done = grp_left == 1;
+            if (!tile_done) {
+                if (!__all_sync(0xffffffffu, next_ready)) ok = mbar_wait_warp(&c->tfull[slot], tph, c, a.status, 2u);
+                tc_fence_after();
+                tmem_ld32(tmem_row + slot * kBN, va);
+            }
             if (DBG) {
                 if (a.acc_debug && row_ok) debug_store<I8>(a, vb, m, n0 + 32, a.Kg - grp_left);
             }
@@ -678,7 +697,15 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
             }
 #pragma unroll
             for (int q = 0; q < 16; ++q) fma2(yacc[16 + q], pack2(vb[2 * q], vb[2 * q + 1]), d2);
-            if (--grp_left == 0 && ok) finish_tile();
+            --grp_left;
+            if (tile_done && ok) {
+                finish_tile();
+                if (ok && more) {
+                    ok = mbar_wait_warp(&c->tfull[slot], tph, c, a.status, 2u);
+                    tc_fence_after();
+                    tmem_ld32(tmem_row + slot * kBN, va);
+                }
+            }
         };
 
         if (total > 0) {

@@ -160,7 +160,9 @@ def test_linear_matches_oracle_small_workloads(tdq, idx):
 
 
 @pytest.mark.parametrize("M,C,O,g", [(1, 32, 8, 32), (129, 64, 65, 32), (300, 96, 200, 32), (257, 320, 130, 32),
-                                     (100, 128, 64, 64), (130, 256, 96, 128), (64, 768, 72, 768), (50, 100, 30, 32)])
+                                     (100, 128, 64, 64), (130, 256, 96, 128), (64, 768, 72, 768), (50, 100, 30, 32),
+                                     # more work items than SMs: a CTA takes several row blocks in turn
+                                     (19200, 32, 128, 32), (2100, 64, 1280, 32), (19100, 64, 100, 64)])
 def test_linear_shapes_tails_bias_and_wide_groups(tdq, M, C, O, g):
     rng = np.random.default_rng(M + C + O)
     x = si.token_mixture(rng, 1, M, C, sigma_log_std=0.5, bg_frac=0.1, bg_nu=3.0, bg_amp=20.0).reshape(-1, C)

@@ -1,0 +1,49 @@
+"""The N > 1 bookkeeping of the benchmark on CPU: two gloo ranks, no GPU.
+
+Rows are independent, so ranks share nothing on the data path; the only cross-rank step is the
+maximum over the ranks' times, from which the whole-job rate is computed."""
+import os
+import socket
+import sys
+
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank, world, port, out):
+    import torch
+    import torch.distributed as dist
+    sys.path.insert(0, ROOT)
+    import bench
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    mine = [10.0 + rank, 3.0 - rank, 7.0]                 # rank 1 is slower on the first, faster on the second
+    got = bench.max_over_ranks(mine, torch.device("cpu"), world)
+    rate = bench.whole_job_rate(1000.0, world, got[0])
+    if rank == 0:
+        out.put((got, rate))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_ranks_take_the_slowest_time_and_sum_the_work():
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got, rate = out.get(timeout=120)
+    for p in procs:
+        p.join(timeout=120)
+        assert p.exitcode == 0
+    assert got == [11.0, 3.0, 7.0]
+    assert abs(rate - 2 * 1000.0 / 11e-3) < 1e-6
