@@ -32,16 +32,16 @@
 //   2. w4a4_gemm_kernel   persistent, one CTA per SM, 128 x 128 output tiles.  Warp roles:
 //        warps 0-1   producers: one lane each issues the bulk copies of alternate ring stages
 //        warp  2     one lane issues the MMAs and the commits that release buffers
-//        warps 4-11  promotion + epilogue: warp w owns TMEM lanes 32 (w % 4).. (its rows) and 64
-//                    columns; a thread keeps 64 float accumulators of one output row
-//      The promotion warps take most of the register file (setmaxnreg): a thread holds its 64
-//      accumulators plus two 32-value landing buffers, so that one TMEM load is in flight while
-//      the FMAs on the other buffer issue.
+//        warps 4-19  promotion + epilogue: warp w owns TMEM lanes 32 (w % 4).. (its rows) and 32
+//                    columns; a thread keeps 32 float accumulators of one output row and one
+//                    32-value landing buffer.  Sixteen warps, four per scheduler: a warp executes
+//                    dependent instructions only every few clocks, so the TMEM load and the
+//                    barrier traffic of one warp hide behind the FMAs of the other three.
 //      A work item is one 128-row block of A with a range of column tiles.  The item's scales,
 //      and its A block when the whole K extent fits, are loaded once per item; B (and A
 //      otherwise) streams through a ring of stages of 4 K-steps.  TMEM holds four 128-column
 //      accumulator slots, each with a full/empty mbarrier pair.
-//      In the epilogue every thread parks its 64 outputs in its own shared-memory strip; the
+//      In the epilogue every thread parks its 32 outputs in its own shared-memory strip; the
 //      promotion warps then read the tile back row by row, so that one warp instruction stores
 //      512 contiguous bytes of y.
 //
@@ -65,17 +65,18 @@ constexpr int kMaxStages = 8;
 constexpr int kProdWarps = 2;
 constexpr int kMmaWarp = 2;
 constexpr int kPromoWarp0 = 4;
-constexpr int kPromoWarps = 8;
-constexpr int kThreads = (kPromoWarp0 + kPromoWarps) * 32;   // 384
-constexpr int kStripBytes = 256;         // one thread's 64 fp32 outputs (128 bytes used for bf16)
+constexpr int kPromoWarps = 16;
+constexpr int kCols = kBN / (kPromoWarps / 4);   // 32 columns of one row per promotion thread
+constexpr int kThreads = (kPromoWarp0 + kPromoWarps) * 32;   // 640
+constexpr int kStripBytes = kCols * 4;   // one thread's 32 fp32 outputs (half of it used for bf16)
 constexpr int kStagingBytes = kPromoWarps * 32 * kStripBytes;
-constexpr int kWsbBytes = kPromoWarps * 512;   // per warp: 64 output-channel scales and 64 biases
+constexpr int kWsbBytes = kPromoWarps * 256;   // per warp: 32 output-channel scales and 32 biases
 constexpr int kCtrlBytes = 256;
 constexpr int kSmemLimit = 232448;       // 227 KB per CTA
 constexpr uint32_t kTmemCols = kSlots * kBN;
 constexpr long long kTimeoutCycles = 2000000000LL;
 constexpr int kExpandThreads = 512;
-constexpr int kRegsControl = 40, kRegsPromo = 232;   // 128 * 40 + 256 * 232 = 384 * 168
+constexpr int kRegsControl = 40, kRegsPromo = 104;   // 128 * 40 + 512 * 104 <= 640 * 96
 
 // instruction descriptors: M = 128, N = 128, both operands K-major
 constexpr uint32_t kIdescShape = ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
@@ -156,6 +157,7 @@ __device__ __forceinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, C
     uint32_t polls = 0;
 #pragma unroll 1
     while (!mbar_try(bar, parity)) {
+        __nanosleep(64);
         if ((++polls & 63u) == 0u) {
             if (c->abort_flag) return false;
             const long long now = clock64();
@@ -226,6 +228,39 @@ __device__ __forceinline__ void mma_issue(uint32_t d_tmem, uint64_t adesc, uint6
             ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(kIdescF8), "r"(accumulate)
             : "memory");
 }
+
+// The same two instructions for a converged warp: every lane executes them, lane 0's predicate lets
+// them through (no branch).  Descriptors are passed as their low words; the high word is constant.
+constexpr uint32_t kDescHi = (256u >> 4) | (1u << 14);   // stride byte offset 256, descriptor version 1
+template <bool I8>
+__device__ __forceinline__ void mma_issue_lane0(int lane, uint32_t d_tmem, uint32_t adesc_lo, uint32_t bdesc_lo,
+                                                uint32_t accumulate) {
+    if (I8)
+        asm volatile(
+            "{\n\t.reg .pred p, q;\n\t.reg .b64 da, db;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\tsetp.eq.s32 q, %5, 0;\n\t"
+            "mov.b64 da, {%1, %6};\n\tmov.b64 db, {%2, %6};\n\t"
+            "@q tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %3, p;\n\t}"
+            ::"r"(d_tmem), "r"(adesc_lo), "r"(bdesc_lo), "r"(kIdescI8), "r"(accumulate), "r"(lane), "r"(kDescHi)
+            : "memory");
+    else
+        asm volatile(
+            "{\n\t.reg .pred p, q;\n\t.reg .b64 da, db;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\tsetp.eq.s32 q, %5, 0;\n\t"
+            "mov.b64 da, {%1, %6};\n\tmov.b64 db, {%2, %6};\n\t"
+            "@q tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], da, db, %3, p;\n\t}"
+            ::"r"(d_tmem), "r"(adesc_lo), "r"(bdesc_lo), "r"(kIdescF8), "r"(accumulate), "r"(lane), "r"(kDescHi)
+            : "memory");
+}
+__device__ __forceinline__ void mma_commit_lane0(int lane, uint32_t bar_s) {
+    asm volatile(
+        "{\n\t.reg .pred q;\n\tsetp.eq.s32 q, %1, 0;\n\t"
+        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+        ::"r"(bar_s), "r"(lane)
+        : "memory");
+}
+// low word of the operand descriptor of a block at shared address saddr (leading byte offset 128)
+__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr) { return ((saddr & 0x3FFFFu) >> 4) | ((128u >> 4) << 16); }
 
 __device__ __forceinline__ void mma_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
@@ -413,16 +448,19 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
 
     if (warp < kPromoWarp0) {
         setmaxnreg_dec<kRegsControl>();
-        if (warp < kProdWarps && lane == 0) {
-            // ------------------------------------------------------------ producers (one lane each)
+        // The control roles run with the whole warp converged and let lane 0 issue: a lone lane whose
+        // warp-mates sit at the final barrier was measured to execute several times slower.
+        if (warp < kProdWarps) {
+            // ------------------------------------------------------------ producers (lane 0 issues)
             uint32_t sc = 0, s = 0, ph = 0, ic = 0;   // stage counter, its ring slot and phase; items so far
             bool ok = true;
             for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++ic) {
                 const int mt = item / a.n_parts, part = item % a.n_parts;
                 const uint8_t* a_src = a.a_blocks + (int64_t)mt * a.n_steps * kBlock;
                 if (warp == 0) {
-                    ok = mbar_wait(&c->a_empty, (ic & 1) ^ 1, c, a.status, 1u);
+                    ok = mbar_wait_warp(&c->a_empty, (ic & 1) ^ 1, c, a.status, 1u);
                     if (!ok) break;
+                    if (lane == 0) {
                     const uint32_t sbytes = (uint32_t)a.Kg * kScaleBlock;
                     mbar_expect_tx(&c->a_full, sbytes + (resident ? (uint32_t)a.n_steps * kBlock : 0u));
                     const uint8_t* s_src = a.s_blocks + (int64_t)mt * a.Kg * kScaleBlock;
@@ -434,13 +472,16 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
                             bulk_load(ares_s + kc * kChunk * kBlock, a_src + (int64_t)kc * kChunk * kBlock,
                                       (uint32_t)nk * kBlock, &c->a_full);
                         }
+                    }
+                    __syncwarp();
                 }
                 for (int nt = part_begin(part); nt < part_begin(part + 1) && ok; ++nt) {
                     const uint8_t* b_src = a.b_blocks + (int64_t)nt * a.n_steps * kBlock;
                     for (int kc = 0; kc < n_chunks; ++kc, ++sc) {
                         if ((int)(sc & 1u) == warp) {
-                            ok = mbar_wait(&c->empty[s], ph ^ 1, c, a.status, 5u);
+                            ok = mbar_wait_warp(&c->empty[s], ph ^ 1, c, a.status, 5u);
                             if (!ok) break;
+                            if (lane == 0) {
                             const int nk = min(kChunk, a.n_steps - kc * kChunk);
                             const uint32_t stage = ring_s + s * a.stage_bytes;
                             mbar_expect_tx(&c->full[s], (uint32_t)nk * kBlock * (resident ? 1u : 2u));
@@ -448,59 +489,72 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
                             if (!resident)
                                 bulk_load(stage + kChunk * kBlock, a_src + (int64_t)kc * kChunk * kBlock,
                                           (uint32_t)nk * kBlock, &c->full[s]);
+                            }
+                            __syncwarp();
                         }
                         if (++s == (uint32_t)a.n_stages) { s = 0; ph ^= 1; }
                     }
                 }
             }
-        } else if (warp == kMmaWarp && lane == 0) {
-            // ------------------------------------------------------------ MMA issue (one lane)
+        } else if (warp == kMmaWarp) {
+            // ------------------------------------------------------------ MMA issue (lane 0 issues)
+            // A warp runs dependent scalar code at one instruction every few clocks, so this loop is
+            // what paces the tensor pipe when promotion is rare: everything that can be is hoisted.
             uint32_t s = 0, ph = 0, slot = 0, tph = 0, ic = 0;
             bool slot_ready = false;   // the early answer about the current slot, if it was yes
-            const uint64_t ares_desc = smem_desc(ares_s);
+            const uint32_t ares_lo = desc_lo(ares_s), ring_lo = desc_lo(ring_s);
+            const uint32_t stage_step = a.stage_bytes >> 4, n_stages = (uint32_t)a.n_stages;
+            const uint32_t a_in_stage = resident ? 0u : (uint32_t)(kChunk * (kBlock >> 4));
+            const uint32_t full_s = smem_u32(&c->full[0]), empty_s = smem_u32(&c->empty[0]);
+            const uint32_t tfull_s = smem_u32(&c->tfull[0]);
+            const int n_steps = a.n_steps;
             bool ok = true;
             for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++ic) {
                 const int part = item % a.n_parts;
-                ok = mbar_wait(&c->a_full, ic & 1, c, a.status, 6u);
-                for (int nt = part_begin(part); nt < part_begin(part + 1) && ok; ++nt) {
-                    int sub = 0, kj = 0;
-                    uint64_t bdesc = 0;
-                    for (int ks = 0; ks < a.n_steps; ++ks) {
-                        if (kj == 0) {
-                            ok = mbar_wait(&c->full[s], ph, c, a.status, 4u);
-                            if (!ok) break;
-                            bdesc = smem_desc(ring_s + s * a.stage_bytes);
+                const int n_tiles = part_begin(part + 1) - part_begin(part);
+                ok = mbar_wait_warp(&c->a_full, ic & 1, c, a.status, 6u);
+                for (int tl = 0; tl < n_tiles && ok; ++tl) {
+                    int sub = 0;
+                    uint32_t a_lo = ares_lo;   // resident: walks through the item's A blocks
+                    for (int k0 = 0; k0 < n_steps && ok; k0 += kChunk) {
+                        ok = mbar_wait_warp(&c->full[s], ph, c, a.status, 4u);
+                        if (!ok) break;
+                        const uint32_t b_lo = ring_lo + s * stage_step;
+                        if (!resident) a_lo = b_lo + a_in_stage;
+                        const int nk = min(kChunk, n_steps - k0);
+#pragma unroll
+                        for (int j = 0; j < kChunk; ++j) {
+                            if (j < nk) {
+                                if (sub == 0 && !slot_ready) {
+                                    ok = mbar_wait_warp(&c->tempty[slot], tph ^ 1, c, a.status, 3u);
+                                    if (!ok) break;
+                                }
+                                const bool last_sub = sub + 1 == spg;
+                                const uint32_t nslot = (slot + 1) & (kSlots - 1), ntph = tph ^ (nslot == 0);
+                                // ask about the next group's slot now: the answer travels while this step is issued
+                                if (last_sub) slot_ready = __all_sync(0xffffffffu, mbar_test(&c->tempty[nslot], ntph ^ 1));
+                                tc_fence_after();
+                                mma_issue_lane0<I8>(lane, tmem_base + slot * kBN, a_lo + j * (kBlock >> 4),
+                                                    b_lo + j * (kBlock >> 4), sub == 0 ? 0u : 1u);
+                                if (last_sub) {
+                                    mma_commit_lane0(lane, tfull_s + slot * 8);
+                                    sub = 0;
+                                    slot = nslot;
+                                    tph = ntph;
+                                } else {
+                                    ++sub;
+                                }
+                            }
                         }
-                        if (sub == 0 && !slot_ready) {
-                            ok = mbar_wait(&c->tempty[slot], tph ^ 1, c, a.status, 3u);
-                            if (!ok) break;
-                        }
-                        // ask about the next group's slot now: the answer travels while this step is issued
-                        const bool last_sub = sub + 1 == spg;
-                        const uint32_t nslot = (slot + 1) & (kSlots - 1), ntph = tph ^ (nslot == 0);
-                        if (last_sub) slot_ready = mbar_test(&c->tempty[nslot], ntph ^ 1);
-                        tc_fence_after();
-                        const uint64_t adesc = resident ? ares_desc + (uint64_t)(ks * (kBlock >> 4))
-                                                        : bdesc + (uint64_t)((kChunk + kj) * (kBlock >> 4));
-                        mma_issue<I8>(tmem_base + slot * kBN, adesc, bdesc + (uint64_t)(kj * (kBlock >> 4)),
-                                      sub == 0 ? 0u : 1u);
-                        if (last_sub) {
-                            sub = 0;
-                            mma_commit(&c->tfull[slot]);
-                            slot = nslot;
-                            tph = ntph;
-                        } else {
-                            ++sub;
-                        }
-                        if (++kj == kChunk || ks == a.n_steps - 1) {
-                            kj = 0;
-                            mma_commit(&c->empty[s]);
-                            if (++s == (uint32_t)a.n_stages) { s = 0; ph ^= 1; }
-                        }
+                        if (!ok) break;
+                        if (resident) a_lo += kChunk * (kBlock >> 4);
+                        mma_commit_lane0(lane, empty_s + s * 8);
+                        if (++s == n_stages) { s = 0; ph ^= 1; }
                     }
                 }
-                if (ok) mma_commit(&c->a_empty);
+                if (ok) mma_commit_lane0(lane, smem_u32(&c->a_empty));
             }
+            (void)full_s;
         }
     } else {
         setmaxnreg_inc<kRegsPromo>();
@@ -508,14 +562,14 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
         const int pw = warp - kPromoWarp0;
         const int quarter = warp & 3;                 // TMEM lanes 32 * quarter .. + 31
         const int row = quarter * 32 + lane;
-        const int col0 = (pw >> 2) * (kBN / 2);
+        const int col0 = (pw >> 2) * kCols;
         const uint32_t tmem_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + col0;
         constexpr int esz = YBF16 ? 2 : 4;
-        constexpr int kChunksPerStrip = 64 * esz / 16;             // 16-byte chunks of one strip
+        constexpr int kChunksPerStrip = kCols * esz / 16;          // 16-byte chunks of one strip
         const uint32_t strips_s = sm_s + a.staging_off;
-        const uint32_t strip_s = strips_s + (uint32_t)(pw * 32 + lane) * kStripBytes;
         const uint32_t swz = (uint32_t)lane & (kChunksPerStrip - 1);   // chunk c of a strip sits at c ^ swz
-        const uint32_t wsb_s = sm_s + a.wsb_off + (uint32_t)pw * 512;
+        const uint32_t strip_s = (strips_s + (uint32_t)(pw * 32 + lane) * kStripBytes) ^ (swz << 4);
+        const uint32_t wsb_s = sm_s + a.wsb_off + (uint32_t)pw * 256;
         const uint32_t my_scale_s = scales_s + (uint32_t)row * 4;
 
         // groups this CTA will see, so that the next slot can be requested early
@@ -525,15 +579,15 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
             total += (uint32_t)(part_begin(part + 1) - part_begin(part)) * (uint32_t)a.Kg;
         }
 
-        uint64_t yacc[kBN / 4];        // 64 floats of one output row, packed in pairs
-        uint32_t va[32], vb[32];       // landing buffers: first and second 32 columns of a slot
+        uint64_t yacc[kCols / 2];      // 32 floats of one output row, packed in pairs
+        uint32_t v[kCols];             // landing buffer: this thread's 32 columns of a slot
 #pragma unroll
-        for (int q = 0; q < 32; ++q) va[q] = vb[q] = 0u;
+        for (int q = 0; q < kCols; ++q) v[q] = 0u;
         uint32_t gc = 0, slot = 0, tph = 0, ic = 0, tc = 0;   // groups, their slot and phase; items, tiles so far
         int item = blockIdx.x, mt = 0, nt = 0, nt_end = 0, grp_left = 0;
         uint32_t scale_s = my_scale_s;   // this row's scale of the group about to be promoted
         int64_t m = 0, n0 = 0;
-        float w0 = 0.f, w1 = 0.f, b0 = 0.f, b1 = 0.f;   // this lane's share of the tile's channel scales and biases
+        float w0 = 0.f, b0 = 0.f;        // this lane's share of the tile's channel scales and biases
         bool ok = true, row_ok = false;
 
         auto begin_item = [&]() {
@@ -550,29 +604,25 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
             grp_left = a.Kg;
             scale_s = my_scale_s;
 #pragma unroll
-            for (int j = 0; j < kBN / 4; ++j) yacc[j] = 0ull;
-            const int64_t ca = n0 + lane, cb = n0 + 32 + lane;
+            for (int j = 0; j < kCols / 2; ++j) yacc[j] = 0ull;
+            const int64_t ca = n0 + lane;
             w0 = ca < a.O ? __ldg(a.wscale + ca) : 0.f;
-            w1 = cb < a.O ? __ldg(a.wscale + cb) : 0.f;
             b0 = (a.bias && ca < a.O) ? __ldg(a.bias + ca) : 0.f;
-            b1 = (a.bias && cb < a.O) ? __ldg(a.bias + cb) : 0.f;
         };
         // y = (s_o * 2^e) * sum + bias for the tile that just finished, then on to the next tile
         auto finish_tile = [&]() {
             sts32(wsb_s + lane * 4, __float_as_uint(__fmul_rn(w0, a.out_scale)));
-            sts32(wsb_s + 128 + lane * 4, __float_as_uint(__fmul_rn(w1, a.out_scale)));
-            sts32(wsb_s + 256 + lane * 4, __float_as_uint(b0));
-            sts32(wsb_s + 384 + lane * 4, __float_as_uint(b1));
+            sts32(wsb_s + 128 + lane * 4, __float_as_uint(b0));
             if (tc > 0)   // the strips of the previous tile have been read by every warp
                 ok = mbar_wait_warp(&c->strips_free, (tc - 1) & 1, c, a.status, 9u);
             __syncwarp();
             if (!ok) return;
 #pragma unroll
-            for (int j = 0; j < kBN / 2; j += 4) {
+            for (int j = 0; j < kCols; j += 4) {
                 float o0, o1, o2, o3;
                 unpack2(yacc[j / 2], o0, o1);
                 unpack2(yacc[j / 2 + 1], o2, o3);
-                const uint4 s4 = lds128(wsb_s + j * 4), b4 = lds128(wsb_s + 256 + j * 4);
+                const uint4 s4 = lds128(wsb_s + j * 4), b4 = lds128(wsb_s + 128 + j * 4);
                 o0 = __fmaf_rn(__uint_as_float(s4.x), o0, __uint_as_float(b4.x));
                 o1 = __fmaf_rn(__uint_as_float(s4.y), o1, __uint_as_float(b4.y));
                 o2 = __fmaf_rn(__uint_as_float(s4.z), o2, __uint_as_float(b4.z));
@@ -581,10 +631,10 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
                     __nv_bfloat162 lo = __floats2bfloat162_rn(o0, o1);
                     __nv_bfloat162 hi = __floats2bfloat162_rn(o2, o3);
                     const uint32_t byte = j * 2;   // 8 bytes inside chunk byte / 16
-                    sts64(strip_s + (((byte >> 4) ^ swz) << 4) + (byte & 15), *reinterpret_cast<uint32_t*>(&lo),
+                    sts64((strip_s ^ ((byte >> 4) << 4)) + (byte & 15), *reinterpret_cast<uint32_t*>(&lo),
                           *reinterpret_cast<uint32_t*>(&hi));
                 } else {
-                    sts128(strip_s + (((uint32_t)(j >> 2) ^ swz) << 4), __float_as_uint(o0), __float_as_uint(o1),
+                    sts128(strip_s ^ ((uint32_t)(j >> 2) << 4), __float_as_uint(o0), __float_as_uint(o1),
                            __float_as_uint(o2), __float_as_uint(o3));
                 }
             }
@@ -592,37 +642,38 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
             mbar_arrive_lane0(&c->strips_ready, lane);
             ok = mbar_wait_warp(&c->strips_ready, tc & 1, c, a.status, 10u);
             if (!ok) return;
-            // warp pw writes tile rows 16 pw .. 16 pw + 15 from the strips
+            // warp pw writes tile rows 8 pw .. 8 pw + 7 from the strips
+            constexpr int kRowsPerWarp = kBM / kPromoWarps;
             if (a.vec_ok) {   // one instruction covers 512 contiguous bytes of y
                 constexpr int kRowsPerInstr = YBF16 ? 2 : 1;       // a tile row is 128 * esz bytes
                 const int sub_row = lane / (32 / kRowsPerInstr);
                 const int chunk = lane % (32 / kRowsPerInstr);     // 16-byte chunk of the tile row
-                const int half = chunk / kChunksPerStrip, cs = chunk % kChunksPerStrip;
+                const int part = chunk / kChunksPerStrip, cs = chunk % kChunksPerStrip;
                 const int64_t col = (int64_t)nt * kBN + chunk * (16 / esz);
-#pragma unroll 4
-                for (int rr = 0; rr < 16; rr += kRowsPerInstr) {
-                    const int r = pw * 16 + rr + sub_row;
+#pragma unroll
+                for (int rr = 0; rr < kRowsPerWarp; rr += kRowsPerInstr) {
+                    const int r = pw * kRowsPerWarp + rr + sub_row;
                     const int64_t mg = (int64_t)mt * kBM + r;
-                    const uint32_t src = strips_s + (uint32_t)((half * 4 + (r >> 5)) * 32 + (r & 31)) * kStripBytes +
+                    const uint32_t src = strips_s + (uint32_t)((part * 4 + (r >> 5)) * 32 + (r & 31)) * kStripBytes +
                                          (((uint32_t)cs ^ ((uint32_t)r & (kChunksPerStrip - 1))) << 4);
                     if (mg < a.M && col < a.O) {
-                        const uint4 v = lds128(src);
+                        const uint4 val = lds128(src);
                         __stcs(reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(a.y) +
-                                                        ((size_t)mg * a.y_stride + col) * esz), v);
+                                                        ((size_t)mg * a.y_stride + col) * esz), val);
                     }
                 }
             } else {          // any alignment: element by element
 #pragma unroll 1
-                for (int rr = 0; rr < 16; ++rr) {
-                    const int r = pw * 16 + rr;
+                for (int rr = 0; rr < kRowsPerWarp; ++rr) {
+                    const int r = pw * kRowsPerWarp + rr;
                     const int64_t mg = (int64_t)mt * kBM + r;
                     if (mg >= a.M) break;
 #pragma unroll 1
                     for (int cc = lane; cc < kBN; cc += 32) {
                         const int64_t col = (int64_t)nt * kBN + cc;
                         if (col >= a.O) break;
-                        const uint32_t byte = (uint32_t)(cc & 63) * esz;
-                        const uint32_t src = strips_s + (uint32_t)(((cc >> 6) * 4 + (r >> 5)) * 32 + (r & 31)) * kStripBytes +
+                        const uint32_t byte = (uint32_t)(cc % kCols) * esz;
+                        const uint32_t src = strips_s + (uint32_t)(((cc / kCols) * 4 + (r >> 5)) * 32 + (r & 31)) * kStripBytes +
                                              (((byte >> 4) ^ ((uint32_t)r & (kChunksPerStrip - 1))) << 4) + (byte & 12u);
                         const uint32_t word = lds32(src);
                         if (YBF16)
@@ -649,63 +700,45 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
             }
             if (ok && item < n_items) begin_tile();
         };
-        // One group.  Its first 32 columns were requested earlier and land in va; request the
-        // second 32 into vb and fold va in meanwhile; then release the slot, request the next
-        // group's first half and fold vb in.  The last request is issued even after the last group
-        // (it re-reads an idle slot) so that the landing buffers are written on every path.
+        // One group: its 32 columns were requested earlier and land in v.  Release the slot as soon as
+        // they have landed, fold them in, then request the next group (after the epilogue at the end
+        // of a tile: the next group may belong to the next work item, which cannot start before this
+        // warp has handed the current item's buffers back).  With four promotion warps per scheduler
+        // the load of one warp hides behind the FMAs of the others.
         auto promote = [&]() {
             const uint32_t dbits = lds32(scale_s);
             scale_s += kScaleBlock;
             const uint64_t d2 = pack2(dbits, dbits);
-            tmem_ld_wait();                               // va has landed
-            tmem_ld32(tmem_row + slot * kBN + 32, vb);
             // ask about the next group's slot now; the answer is needed only after the FMAs below
             const uint32_t nslot = (slot + 1) & (kSlots - 1), ntph = tph ^ (nslot == 0);
             const bool more = gc + 1 < total;
             const bool next_ready = more ? mbar_test(&c->tfull[nslot], ntph) : true;
-            if (DBG) {
-                if (a.acc_debug && row_ok) debug_store<I8>(a, va, m, n0, a.Kg - grp_left);
-            }
-            if (I8) {
-#pragma unroll
-                for (int q = 0; q < 32; ++q) va[q] = __float_as_uint((float)(int32_t)va[q]);
-            }
-#pragma unroll
-            for (int q = 0; q < 16; ++q) fma2(yacc[q], pack2(va[2 * q], va[2 * q + 1]), d2);
-            tmem_ld_wait();                               // vb has landed: the slot is drained
+            tmem_ld_wait();                               // v has landed: the slot is drained
             tc_fence_before();
             __syncwarp();
             mbar_arrive_lane0(&c->tempty[slot], lane);
             slot = nslot;
             tph = ntph;
             ++gc;
-            // Request the next group's first half before folding vb in, except at the end of a tile:
-            // there the epilogue goes first, because the next group may belong to the next work item,
-            // which cannot start before this warp has handed the current item's buffers back.
-            const bool tile_done = grp_left == 1;
-            if (!tile_done) {
-                if (!__all_sync(0xffffffffu, next_ready)) ok = mbar_wait_warp(&c->tfull[slot], tph, c, a.status, 2u);
-                tc_fence_after();
-                tmem_ld32(tmem_row + slot * kBN, va);
-            }
             if (DBG) {
-                if (a.acc_debug && row_ok) debug_store<I8>(a, vb, m, n0 + 32, a.Kg - grp_left);
+                if (a.acc_debug && row_ok) debug_store<I8>(a, v, m, n0, a.Kg - grp_left);
             }
             if (I8) {
 #pragma unroll
-                for (int q = 0; q < 32; ++q) vb[q] = __float_as_uint((float)(int32_t)vb[q]);
+                for (int q = 0; q < kCols; ++q) v[q] = __float_as_uint((float)(int32_t)v[q]);
             }
 #pragma unroll
-            for (int q = 0; q < 16; ++q) fma2(yacc[16 + q], pack2(vb[2 * q], vb[2 * q + 1]), d2);
-            --grp_left;
-            if (tile_done && ok) {
+            for (int q = 0; q < kCols / 2; ++q) fma2(yacc[q], pack2(v[2 * q], v[2 * q + 1]), d2);
+            const bool tile_done = --grp_left == 0;
+            if (tile_done) {
                 finish_tile();
-                if (ok && more) {
-                    ok = mbar_wait_warp(&c->tfull[slot], tph, c, a.status, 2u);
-                    tc_fence_after();
-                    tmem_ld32(tmem_row + slot * kBN, va);
-                }
+                if (!ok || !more) return;
+                ok = mbar_wait_warp(&c->tfull[slot], tph, c, a.status, 2u);
+            } else if (!__all_sync(0xffffffffu, next_ready)) {
+                ok = mbar_wait_warp(&c->tfull[slot], tph, c, a.status, 2u);
             }
+            tc_fence_after();
+            tmem_ld32(tmem_row + slot * kBN, v);
         };
 
         if (total > 0) {
@@ -715,7 +748,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
                 ok = mbar_wait_warp(&c->tfull[0], 0, c, a.status, 2u);
             }
             tc_fence_after();
-            tmem_ld32(tmem_row, va);
+            tmem_ld32(tmem_row, v);
 #pragma unroll 1
             while (ok && gc < total) promote();
         }
