@@ -185,6 +185,27 @@ __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, C
     return __all_sync(0xffffffffu, mbar_wait_slow(bar, parity, c, status, code));
 }
 
+// The same primitives on 32-bit shared-window addresses, for the hot loops (no pointer conversion).
+__device__ __forceinline__ bool mbar_test_s(uint32_t bar_s, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar_s), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void mbar_arrive_lane0_s(uint32_t bar_s, int lane) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.eq.s32 p, %1, 0;\n\t"
+        "@p mbarrier.arrive.shared::cta.b64 _, [%0];\n\t}"
+        ::"r"(bar_s), "r"(lane)
+        : "memory");
+}
+
 // lane 0 of a converged warp arrives; predicated, so the warp does not diverge
 __device__ __forceinline__ void mbar_arrive_lane0(uint64_t* bar, int lane) {
     asm volatile(
@@ -410,10 +431,9 @@ __device__ __noinline__ void debug_store(const LinArgs& a, const uint32_t* v, in
 
 template <bool I8, bool YBF16, bool DBG>
 __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
-    Ctrl* c = reinterpret_cast<Ctrl*>(sm);
-    const uint32_t sm_s = smem_u32(sm);
+    extern __shared__ __align__(128) uint8_t smem_raw[];   // no static shared memory: the window starts aligned
+    Ctrl* c = reinterpret_cast<Ctrl*>(smem_raw);
+    const uint32_t sm_s = smem_u32(smem_raw);
     const uint32_t scales_s = sm_s + kCtrlBytes;        // [Kg][128] floats of the item
     const uint32_t ares_s = sm_s + a.ares_off;          // [n_steps] operand blocks of the item, if resident
     const uint32_t ring_s = sm_s + a.ring_off;
@@ -705,6 +725,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
         // of a tile: the next group may belong to the next work item, which cannot start before this
         // warp has handed the current item's buffers back).  With four promotion warps per scheduler
         // the load of one warp hides behind the FMAs of the others.
+        const uint32_t tfull_s = smem_u32(&c->tfull[0]), tempty_s = smem_u32(&c->tempty[0]);
         auto promote = [&]() {
             const uint32_t dbits = lds32(scale_s);
             scale_s += kScaleBlock;
@@ -712,14 +733,11 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
             // ask about the next group's slot now; the answer is needed only after the FMAs below
             const uint32_t nslot = (slot + 1) & (kSlots - 1), ntph = tph ^ (nslot == 0);
             const bool more = gc + 1 < total;
-            const bool next_ready = more ? mbar_test(&c->tfull[nslot], ntph) : true;
+            const bool next_ready = mbar_test_s(tfull_s + nslot * 8, ntph) || !more;
             tmem_ld_wait();                               // v has landed: the slot is drained
             tc_fence_before();
             __syncwarp();
-            mbar_arrive_lane0(&c->tempty[slot], lane);
-            slot = nslot;
-            tph = ntph;
-            ++gc;
+            mbar_arrive_lane0_s(tempty_s + slot * 8, lane);
             if (DBG) {
                 if (a.acc_debug && row_ok) debug_store<I8>(a, v, m, n0, a.Kg - grp_left);
             }
@@ -729,8 +747,10 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
             }
 #pragma unroll
             for (int q = 0; q < kCols / 2; ++q) fma2(yacc[q], pack2(v[2 * q], v[2 * q + 1]), d2);
-            const bool tile_done = --grp_left == 0;
-            if (tile_done) {
+            slot = nslot;
+            tph = ntph;
+            ++gc;
+            if (--grp_left == 0) {
                 finish_tile();
                 if (!ok || !more) return;
                 ok = mbar_wait_warp(&c->tfull[slot], tph, c, a.status, 2u);
