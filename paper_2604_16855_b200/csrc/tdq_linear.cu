@@ -49,6 +49,7 @@
 // workspace status word and raises a CTA-wide flag; every role then leaves its loops, the CTA
 // releases its TMEM and returns.
 #include <mutex>
+#include <type_traits>
 
 #include "tdq_common.cuh"
 
@@ -441,10 +442,11 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
     const bool resident = a.a_resident != 0;
 
     if (t == 0) {
-        for (int i = 0; i < kMaxStages; ++i) { mbar_init(&c->full[i], 1); mbar_init(&c->empty[i], 1); }
+        const uint32_t n_issuers = a.steps_per_grp == 1 ? 2u : 1u;   // MMA-issuing warps
+        for (int i = 0; i < kMaxStages; ++i) { mbar_init(&c->full[i], 1); mbar_init(&c->empty[i], n_issuers); }
         for (int i = 0; i < kSlots; ++i) { mbar_init(&c->tfull[i], 1); mbar_init(&c->tempty[i], kPromoWarps); }
         mbar_init(&c->a_full, 1);
-        mbar_init(&c->a_empty, 1 + kPromoWarps);
+        mbar_init(&c->a_empty, n_issuers + kPromoWarps);
         mbar_init(&c->strips_ready, kPromoWarps);
         mbar_init(&c->strips_free, kPromoWarps);
         c->abort_flag = 0;
@@ -516,65 +518,86 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
                     }
                 }
             }
-        } else if (warp == kMmaWarp) {
+        } else if (warp == kMmaWarp || spg == 1) {
             // ------------------------------------------------------------ MMA issue (lane 0 issues)
             // A warp runs dependent scalar code at one instruction every few clocks, so this loop is
-            // what paces the tensor pipe when promotion is rare: everything that can be is hoisted.
-            uint32_t s = 0, ph = 0, slot = 0, tph = 0, ic = 0;
-            bool slot_ready = false;   // the early answer about the current slot, if it was yes
+            // what paces the tensor pipe: everything that can be is hoisted, and the two cases are
+            // compiled separately.  With one instruction per group (g = 32) the groups are
+            // independent and two warps take them in turn (even and odd slots), so that each has two
+            // groups' time for its bookkeeping; wider groups chain into one slot and stay with one warp.
+            const uint32_t me = (uint32_t)(warp - kMmaWarp);
             const uint32_t ares_lo = desc_lo(ares_s), ring_lo = desc_lo(ring_s);
             const uint32_t stage_step = a.stage_bytes >> 4, n_stages = (uint32_t)a.n_stages;
             const uint32_t a_in_stage = resident ? 0u : (uint32_t)(kChunk * (kBlock >> 4));
-            const uint32_t full_s = smem_u32(&c->full[0]), empty_s = smem_u32(&c->empty[0]);
-            const uint32_t tfull_s = smem_u32(&c->tfull[0]);
+            const uint32_t empty_s = smem_u32(&c->empty[0]), tfull_s = smem_u32(&c->tfull[0]);
+            const uint32_t tempty_s = smem_u32(&c->tempty[0]);
             const int n_steps = a.n_steps;
-            bool ok = true;
-            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++ic) {
-                const int part = item % a.n_parts;
-                const int n_tiles = part_begin(part + 1) - part_begin(part);
-                ok = mbar_wait_warp(&c->a_full, ic & 1, c, a.status, 6u);
-                for (int tl = 0; tl < n_tiles && ok; ++tl) {
-                    int sub = 0;
-                    uint32_t a_lo = ares_lo;   // resident: walks through the item's A blocks
-                    for (int k0 = 0; k0 < n_steps && ok; k0 += kChunk) {
-                        ok = mbar_wait_warp(&c->full[s], ph, c, a.status, 4u);
-                        if (!ok) break;
-                        const uint32_t b_lo = ring_lo + s * stage_step;
-                        if (!resident) a_lo = b_lo + a_in_stage;
-                        const int nk = min(kChunk, n_steps - k0);
+            auto role = [&](auto dual_tag) {
+                constexpr bool DUAL = decltype(dual_tag)::value;
+                uint32_t s = 0, ph = 0, slot = 0, tph = 0, ic = 0;
+                bool slot_ready = false;   // the early answer about this warp's next slot, if it was yes
+                bool ok = true;
+                for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++ic) {
+                    const int part = item % a.n_parts;
+                    const int n_tiles = part_begin(part + 1) - part_begin(part);
+                    ok = mbar_wait_warp(&c->a_full, ic & 1, c, a.status, 6u);
+                    for (int tl = 0; tl < n_tiles && ok; ++tl) {
+                        int sub = 0;
+                        uint32_t a_lo = ares_lo;   // resident: walks through the item's A blocks
+                        for (int k0 = 0; k0 < n_steps && ok; k0 += kChunk) {
+                            ok = mbar_wait_warp(&c->full[s], ph, c, a.status, 4u);
+                            if (!ok) break;
+                            const uint32_t b_lo = ring_lo + s * stage_step;
+                            if (!resident) a_lo = b_lo + a_in_stage;
+                            const int nk = min(kChunk, n_steps - k0);
 #pragma unroll
-                        for (int j = 0; j < kChunk; ++j) {
-                            if (j < nk) {
-                                if (sub == 0 && !slot_ready) {
-                                    ok = mbar_wait_warp(&c->tempty[slot], tph ^ 1, c, a.status, 3u);
-                                    if (!ok) break;
-                                }
-                                const bool last_sub = sub + 1 == spg;
-                                const uint32_t nslot = (slot + 1) & (kSlots - 1), ntph = tph ^ (nslot == 0);
-                                // ask about the next group's slot now: the answer travels while this step is issued
-                                if (last_sub) slot_ready = __all_sync(0xffffffffu, mbar_test(&c->tempty[nslot], ntph ^ 1));
-                                tc_fence_after();
-                                mma_issue_lane0<I8>(lane, tmem_base + slot * kBN, a_lo + j * (kBlock >> 4),
-                                                    b_lo + j * (kBlock >> 4), sub == 0 ? 0u : 1u);
-                                if (last_sub) {
-                                    mma_commit_lane0(lane, tfull_s + slot * 8);
-                                    sub = 0;
-                                    slot = nslot;
-                                    tph = ntph;
-                                } else {
-                                    ++sub;
+                            for (int j = 0; j < kChunk; ++j) {
+                                if (j < nk) {
+                                    if (DUAL) {
+                                        if ((slot & 1u) == me) {
+                                            if (!slot_ready) {
+                                                ok = mbar_wait_warp(&c->tempty[slot], tph ^ 1, c, a.status, 3u);
+                                                if (!ok) break;
+                                            }
+                                            // ask about this warp's next slot now: the answer travels while this step is issued
+                                            slot_ready = __all_sync(0xffffffffu, mbar_test_s(tempty_s + (slot ^ 2u) * 8,
+                                                                                             tph ^ (slot >> 1) ^ 1u));
+                                            tc_fence_after();
+                                            mma_issue_lane0<I8>(lane, tmem_base + slot * kBN, a_lo + j * (kBlock >> 4),
+                                                                b_lo + j * (kBlock >> 4), 0u);
+                                            mma_commit_lane0(lane, tfull_s + slot * 8);
+                                        }
+                                        slot = (slot + 1) & (kSlots - 1);
+                                        tph ^= (slot == 0);
+                                    } else {
+                                        if (sub == 0 && !slot_ready) {
+                                            ok = mbar_wait_warp(&c->tempty[slot], tph ^ 1, c, a.status, 3u);
+                                            if (!ok) break;
+                                        }
+                                        tc_fence_after();
+                                        mma_issue_lane0<I8>(lane, tmem_base + slot * kBN, a_lo + j * (kBlock >> 4),
+                                                            b_lo + j * (kBlock >> 4), sub == 0 ? 0u : 1u);
+                                        if (++sub == spg) {
+                                            sub = 0;
+                                            mma_commit_lane0(lane, tfull_s + slot * 8);
+                                            slot = (slot + 1) & (kSlots - 1);
+                                            tph ^= (slot == 0);
+                                            slot_ready = __all_sync(0xffffffffu, mbar_test_s(tempty_s + slot * 8, tph ^ 1u));
+                                        }
+                                    }
                                 }
                             }
+                            if (!ok) break;
+                            if (resident) a_lo += kChunk * (kBlock >> 4);
+                            mma_commit_lane0(lane, empty_s + s * 8);
+                            if (++s == n_stages) { s = 0; ph ^= 1; }
                         }
-                        if (!ok) break;
-                        if (resident) a_lo += kChunk * (kBlock >> 4);
-                        mma_commit_lane0(lane, empty_s + s * 8);
-                        if (++s == n_stages) { s = 0; ph ^= 1; }
                     }
+                    if (ok) mma_commit_lane0(lane, smem_u32(&c->a_empty));
                 }
-                if (ok) mma_commit_lane0(lane, smem_u32(&c->a_empty));
-            }
-            (void)full_s;
+            };
+            if (spg == 1) role(std::true_type{});
+            else role(std::false_type{});
         }
     } else {
         setmaxnreg_inc<kRegsPromo>();
