@@ -69,9 +69,8 @@ constexpr int kPromoWarp0 = 4;
 constexpr int kPromoWarps = 16;
 constexpr int kCols = kBN / (kPromoWarps / 4);   // 32 columns of one row per promotion thread
 constexpr int kThreads = (kPromoWarp0 + kPromoWarps) * 32;   // 640
-constexpr int kStripBytes = kCols * 4;   // one thread's 32 fp32 outputs (half of it used for bf16)
+constexpr int kStripBytes = kCols * 4;   // one thread's 32 raw fp32 sums
 constexpr int kStagingBytes = kPromoWarps * 32 * kStripBytes;
-constexpr int kWsbBytes = kPromoWarps * 256;   // per warp: 32 output-channel scales and 32 biases
 constexpr int kCtrlBytes = 256;
 constexpr int kSmemLimit = 232448;       // 227 KB per CTA
 constexpr uint32_t kTmemCols = kSlots * kBN;
@@ -97,7 +96,7 @@ struct LinArgs {
     int32_t tiles_m, tiles_n, n_parts;
     int32_t a_resident;        // the item's whole A block stays in shared memory
     int32_t n_stages;
-    uint32_t ares_off, ring_off, stage_bytes, staging_off, wsb_off;   // shared-memory carve-up
+    uint32_t ares_off, ring_off, stage_bytes, staging_off;   // shared-memory carve-up
     void* y;
     int64_t y_stride;
     int32_t* acc_debug;
@@ -110,7 +109,6 @@ struct Ctrl {
     uint64_t full[kMaxStages], empty[kMaxStages];
     uint64_t tfull[kSlots], tempty[kSlots];
     uint64_t a_full, a_empty;
-    uint64_t strips_ready, strips_free;   // epilogue hand-over between the promotion warps
     uint32_t tmem_base;
     volatile int abort_flag;
 };
@@ -447,8 +445,6 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
         for (int i = 0; i < kSlots; ++i) { mbar_init(&c->tfull[i], 1); mbar_init(&c->tempty[i], kPromoWarps); }
         mbar_init(&c->a_full, 1);
         mbar_init(&c->a_empty, n_issuers + kPromoWarps);
-        mbar_init(&c->strips_ready, kPromoWarps);
-        mbar_init(&c->strips_free, kPromoWarps);
         c->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -607,13 +603,21 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
         const int row = quarter * 32 + lane;
         const int col0 = (pw >> 2) * kCols;
         const uint32_t tmem_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + col0;
+        // Epilogue geometry.  A warp owns one 32 x 32 block of every tile (the rows of its TMEM lanes,
+        // its 32 columns) and needs no other warp to write it out: it parks the raw sums in 4 KB of
+        // shared memory of its own, one 128-byte row per lane, and reads them back with kLPR lanes per
+        // row, so that a store instruction writes whole 128-byte (fp32) or 64-byte (bf16) row segments.
+        // On the way back a lane always meets the same columns and keeps their scales in registers.
         constexpr int esz = YBF16 ? 2 : 4;
-        constexpr int kChunksPerStrip = kCols * esz / 16;          // 16-byte chunks of one strip
-        const uint32_t strips_s = sm_s + a.staging_off;
-        const uint32_t swz = (uint32_t)lane & (kChunksPerStrip - 1);   // chunk c of a strip sits at c ^ swz
-        const uint32_t strip_s = (strips_s + (uint32_t)(pw * 32 + lane) * kStripBytes) ^ (swz << 4);
-        const uint32_t wsb_s = sm_s + a.wsb_off + (uint32_t)pw * 256;
+        constexpr int kLPR = YBF16 ? 4 : 8;           // lanes per row on the way out
+        constexpr int kRPI = 32 / kLPR;               // rows per store instruction
+        constexpr int kCPL = kCols / kLPR;            // columns per lane: 16 bytes of y
+        const int sub = lane / kLPR, cl = lane % kLPR;
+        const uint32_t strip_w = sm_s + a.staging_off + (uint32_t)pw * (32 * kStripBytes);
+        // 16-byte chunk j of row r sits at chunk position j ^ (r & 7): conflict-free both ways
+        const uint32_t strip_wr = (strip_w + (uint32_t)lane * kStripBytes) ^ (((uint32_t)lane & 7u) << 4);
         const uint32_t my_scale_s = scales_s + (uint32_t)row * 4;
+        const size_t row_step = (size_t)kRPI * (size_t)a.y_stride * esz;
 
         // groups this CTA will see, so that the next slot can be requested early
         uint32_t total = 0;
@@ -626,12 +630,13 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
         uint32_t v[kCols];             // landing buffer: this thread's 32 columns of a slot
 #pragma unroll
         for (int q = 0; q < kCols; ++q) v[q] = 0u;
-        uint32_t gc = 0, slot = 0, tph = 0, ic = 0, tc = 0;   // groups, their slot and phase; items, tiles so far
+        uint32_t gc = 0, slot = 0, tph = 0, ic = 0;   // groups, their slot and phase; items so far
         int item = blockIdx.x, mt = 0, nt = 0, nt_end = 0, grp_left = 0;
         uint32_t scale_s = my_scale_s;   // this row's scale of the group about to be promoted
         int64_t m = 0, n0 = 0;
-        float w0 = 0.f, b0 = 0.f;        // this lane's share of the tile's channel scales and biases
-        bool ok = true, row_ok = false;
+        int rows_left = 0;               // rows of y from this lane's first output row to the end
+        float ws[kCPL], bs[kCPL];        // s_o * 2^e and bias of the columns this lane writes
+        bool ok = true, row_ok = false, col_ok = false;
 
         auto begin_item = [&]() {
             mt = item / a.n_parts;
@@ -640,6 +645,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
             nt_end = part_begin(part + 1);
             m = (int64_t)mt * kBM + row;
             row_ok = m < a.M;
+            const int64_t m_out = (int64_t)mt * kBM + quarter * 32 + (a.vec_ok ? sub : 0);
+            rows_left = (int)min((int64_t)32, max((int64_t)0, a.M - m_out));
             ok = mbar_wait_warp(&c->a_full, ic & 1, c, a.status, 7u);
         };
         auto begin_tile = [&]() {
@@ -648,88 +655,75 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
             scale_s = my_scale_s;
 #pragma unroll
             for (int j = 0; j < kCols / 2; ++j) yacc[j] = 0ull;
-            const int64_t ca = n0 + lane;
-            w0 = ca < a.O ? __ldg(a.wscale + ca) : 0.f;
-            b0 = (a.bias && ca < a.O) ? __ldg(a.bias + ca) : 0.f;
+            // vector stores: this lane writes columns n0 + cl * kCPL ...; otherwise column n0 + lane
+            const int64_t cb = n0 + (a.vec_ok ? cl * kCPL : lane);
+            col_ok = cb < a.O;
+#pragma unroll
+            for (int e = 0; e < kCPL; ++e) {
+                const bool in = cb + e < a.O && (a.vec_ok || e == 0);
+                ws[e] = in ? __fmul_rn(__ldg(a.wscale + cb + e), a.out_scale) : 0.f;
+                bs[e] = (in && a.bias) ? __ldg(a.bias + cb + e) : 0.f;
+            }
         };
         // y = (s_o * 2^e) * sum + bias for the tile that just finished, then on to the next tile
         auto finish_tile = [&]() {
-            sts32(wsb_s + lane * 4, __float_as_uint(__fmul_rn(w0, a.out_scale)));
-            sts32(wsb_s + 128 + lane * 4, __float_as_uint(b0));
-            if (tc > 0)   // the strips of the previous tile have been read by every warp
-                ok = mbar_wait_warp(&c->strips_free, (tc - 1) & 1, c, a.status, 9u);
-            __syncwarp();
-            if (!ok) return;
 #pragma unroll
-            for (int j = 0; j < kCols; j += 4) {
+            for (int j = 0; j < kCols / 4; ++j) {
                 float o0, o1, o2, o3;
-                unpack2(yacc[j / 2], o0, o1);
-                unpack2(yacc[j / 2 + 1], o2, o3);
-                const uint4 s4 = lds128(wsb_s + j * 4), b4 = lds128(wsb_s + 128 + j * 4);
-                o0 = __fmaf_rn(__uint_as_float(s4.x), o0, __uint_as_float(b4.x));
-                o1 = __fmaf_rn(__uint_as_float(s4.y), o1, __uint_as_float(b4.y));
-                o2 = __fmaf_rn(__uint_as_float(s4.z), o2, __uint_as_float(b4.z));
-                o3 = __fmaf_rn(__uint_as_float(s4.w), o3, __uint_as_float(b4.w));
-                if (YBF16) {
-                    __nv_bfloat162 lo = __floats2bfloat162_rn(o0, o1);
-                    __nv_bfloat162 hi = __floats2bfloat162_rn(o2, o3);
-                    const uint32_t byte = j * 2;   // 8 bytes inside chunk byte / 16
-                    sts64((strip_s ^ ((byte >> 4) << 4)) + (byte & 15), *reinterpret_cast<uint32_t*>(&lo),
-                          *reinterpret_cast<uint32_t*>(&hi));
-                } else {
-                    sts128(strip_s ^ ((uint32_t)(j >> 2) << 4), __float_as_uint(o0), __float_as_uint(o1),
-                           __float_as_uint(o2), __float_as_uint(o3));
-                }
+                unpack2(yacc[2 * j], o0, o1);
+                unpack2(yacc[2 * j + 1], o2, o3);
+                sts128(strip_wr ^ ((uint32_t)j << 4), __float_as_uint(o0), __float_as_uint(o1), __float_as_uint(o2),
+                       __float_as_uint(o3));
             }
             __syncwarp();
-            mbar_arrive_lane0(&c->strips_ready, lane);
-            ok = mbar_wait_warp(&c->strips_ready, tc & 1, c, a.status, 10u);
-            if (!ok) return;
-            // warp pw writes tile rows 8 pw .. 8 pw + 7 from the strips
-            constexpr int kRowsPerWarp = kBM / kPromoWarps;
-            if (a.vec_ok) {   // one instruction covers 512 contiguous bytes of y
-                constexpr int kRowsPerInstr = YBF16 ? 2 : 1;       // a tile row is 128 * esz bytes
-                const int sub_row = lane / (32 / kRowsPerInstr);
-                const int chunk = lane % (32 / kRowsPerInstr);     // 16-byte chunk of the tile row
-                const int part = chunk / kChunksPerStrip, cs = chunk % kChunksPerStrip;
-                const int64_t col = (int64_t)nt * kBN + chunk * (16 / esz);
+            if (a.vec_ok) {
+                uint8_t* dst = reinterpret_cast<uint8_t*>(a.y) +
+                               ((size_t)((int64_t)mt * kBM + quarter * 32 + sub) * a.y_stride + (size_t)(n0 + cl * kCPL)) * esz;
 #pragma unroll
-                for (int rr = 0; rr < kRowsPerWarp; rr += kRowsPerInstr) {
-                    const int r = pw * kRowsPerWarp + rr + sub_row;
-                    const int64_t mg = (int64_t)mt * kBM + r;
-                    const uint32_t src = strips_s + (uint32_t)((part * 4 + (r >> 5)) * 32 + (r & 31)) * kStripBytes +
-                                         (((uint32_t)cs ^ ((uint32_t)r & (kChunksPerStrip - 1))) << 4);
-                    if (mg < a.M && col < a.O) {
-                        const uint4 val = lds128(src);
-                        __stcs(reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(a.y) +
-                                                        ((size_t)mg * a.y_stride + col) * esz), val);
+                for (int it = 0; it < kLPR; ++it) {
+                    const uint32_t r = (uint32_t)(it * kRPI + sub);
+                    float o[kCPL];
+#pragma unroll
+                    for (int e4 = 0; e4 < kCPL / 4; ++e4) {
+                        const uint32_t ch = (uint32_t)(cl * (kCPL / 4) + e4);
+                        const uint4 q = lds128(strip_w + r * kStripBytes + ((ch ^ (r & 7u)) << 4));
+                        o[4 * e4 + 0] = __fmaf_rn(ws[4 * e4 + 0], __uint_as_float(q.x), bs[4 * e4 + 0]);
+                        o[4 * e4 + 1] = __fmaf_rn(ws[4 * e4 + 1], __uint_as_float(q.y), bs[4 * e4 + 1]);
+                        o[4 * e4 + 2] = __fmaf_rn(ws[4 * e4 + 2], __uint_as_float(q.z), bs[4 * e4 + 2]);
+                        o[4 * e4 + 3] = __fmaf_rn(ws[4 * e4 + 3], __uint_as_float(q.w), bs[4 * e4 + 3]);
+                    }
+                    if (it * kRPI < rows_left && col_ok) {
+                        uint4 val;
+                        if (YBF16) {
+                            __nv_bfloat162 h0 = __floats2bfloat162_rn(o[0], o[1]);
+                            __nv_bfloat162 h1 = __floats2bfloat162_rn(o[2], o[3]);
+                            __nv_bfloat162 h2 = __floats2bfloat162_rn(o[kCPL - 4], o[kCPL - 3]);
+                            __nv_bfloat162 h3 = __floats2bfloat162_rn(o[kCPL - 2], o[kCPL - 1]);
+                            val = make_uint4(*reinterpret_cast<uint32_t*>(&h0), *reinterpret_cast<uint32_t*>(&h1),
+                                             *reinterpret_cast<uint32_t*>(&h2), *reinterpret_cast<uint32_t*>(&h3));
+                        } else {
+                            val = make_uint4(__float_as_uint(o[0]), __float_as_uint(o[1]), __float_as_uint(o[2]),
+                                             __float_as_uint(o[3]));
+                        }
+                        __stcs(reinterpret_cast<uint4*>(dst + (size_t)it * row_step), val);
                     }
                 }
-            } else {          // any alignment: element by element
+            } else {          // any alignment: a row at a time, lane = column
 #pragma unroll 1
-                for (int rr = 0; rr < kRowsPerWarp; ++rr) {
-                    const int r = pw * kRowsPerWarp + rr;
-                    const int64_t mg = (int64_t)mt * kBM + r;
-                    if (mg >= a.M) break;
-#pragma unroll 1
-                    for (int cc = lane; cc < kBN; cc += 32) {
-                        const int64_t col = (int64_t)nt * kBN + cc;
-                        if (col >= a.O) break;
-                        const uint32_t byte = (uint32_t)(cc % kCols) * esz;
-                        const uint32_t src = strips_s + (uint32_t)(((cc / kCols) * 4 + (r >> 5)) * 32 + (r & 31)) * kStripBytes +
-                                             (((byte >> 4) ^ ((uint32_t)r & (kChunksPerStrip - 1))) << 4) + (byte & 12u);
-                        const uint32_t word = lds32(src);
+                for (int r = 0; r < rows_left; ++r) {
+                    const uint32_t word = lds32(strip_w + (uint32_t)r * kStripBytes +
+                                                ((((uint32_t)lane >> 2) ^ ((uint32_t)r & 7u)) << 4) + ((uint32_t)lane & 3u) * 4);
+                    const float o = __fmaf_rn(ws[0], __uint_as_float(word), bs[0]);
+                    const int64_t mg = (int64_t)mt * kBM + quarter * 32 + r;
+                    if (col_ok) {
                         if (YBF16)
-                            reinterpret_cast<uint16_t*>(a.y)[mg * a.y_stride + col] =
-                                (uint16_t)((byte & 2) ? (word >> 16) : (word & 0xffffu));
+                            reinterpret_cast<__nv_bfloat16*>(a.y)[mg * a.y_stride + n0 + lane] = __float2bfloat16_rn(o);
                         else
-                            reinterpret_cast<uint32_t*>(a.y)[mg * a.y_stride + col] = word;
+                            reinterpret_cast<float*>(a.y)[mg * a.y_stride + n0 + lane] = o;
                     }
                 }
             }
-            __syncwarp();
-            mbar_arrive_lane0(&c->strips_free, lane);
-            ++tc;
+            __syncwarp();     // the strip may be overwritten by the next tile
             // next tile, next item
             if (++nt == nt_end) {
                 // the item's scales were read through the generic proxy; the next item's bulk copies
@@ -815,7 +809,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
 struct Plan {
     int64_t tiles_m, tiles_n;
     int32_t n_steps, n_chunks, Kg, n_parts, a_resident, n_stages;
-    uint32_t ares_off, ring_off, stage_bytes, staging_off, wsb_off, smem_bytes;
+    uint32_t ares_off, ring_off, stage_bytes, staging_off, smem_bytes;
     size_t a_bytes, b_bytes, s_bytes;   // operand and scale blocks in the workspace
 };
 
@@ -834,7 +828,7 @@ bool make_plan(int64_t M, int64_t I_pad, int64_t O, int32_t g, int n_sm, Plan& p
     p.s_bytes = (size_t)p.tiles_m * p.Kg * kScaleBlock;
     // shared memory: control, the item's scales, [resident A], ring, output strips, channel scales
     const int64_t scales = (int64_t)p.Kg * kScaleBlock;
-    const int64_t fixed = 128 + kCtrlBytes + scales + kStagingBytes + kWsbBytes;
+    const int64_t fixed = 128 + kCtrlBytes + scales + kStagingBytes;
     const int64_t a_res = (int64_t)p.n_steps * kBlock;
     const int64_t stage_b = (int64_t)kChunk * kBlock, stage_ab = 2 * stage_b;
     const int64_t stages_res = (kSmemLimit - fixed - a_res) / stage_b;
@@ -853,8 +847,7 @@ bool make_plan(int64_t M, int64_t I_pad, int64_t O, int32_t g, int n_sm, Plan& p
         p.ring_off = p.ares_off;
     }
     p.staging_off = p.ring_off + (uint32_t)p.n_stages * p.stage_bytes;
-    p.wsb_off = p.staging_off + kStagingBytes;
-    p.smem_bytes = p.wsb_off + kWsbBytes + 128;
+    p.smem_bytes = p.staging_off + kStagingBytes + 128;
     // split the column tiles of a row block into parts so that the items fill the SMs evenly
     int best = 1;
     int64_t best_cost = INT64_MAX;
@@ -938,7 +931,7 @@ extern "C" tdq_status tdq_w4a4_linear(const uint8_t* xcodes, const float* xscale
     a.tiles_m = e.tiles_m; a.tiles_n = e.tiles_n; a.n_parts = p.n_parts;
     a.a_resident = p.a_resident; a.n_stages = p.n_stages;
     a.ares_off = p.ares_off; a.ring_off = p.ring_off; a.stage_bytes = p.stage_bytes;
-    a.staging_off = p.staging_off; a.wsb_off = p.wsb_off;
+    a.staging_off = p.staging_off;
     a.y = y; a.y_stride = y_row_stride; a.acc_debug = acc_debug;
     a.status = reinterpret_cast<uint32_t*>(workspace);
     const int64_t esz = y_dtype == TDQ_BF16 ? 2 : 4;
