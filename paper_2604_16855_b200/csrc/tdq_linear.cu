@@ -249,34 +249,35 @@ __device__ __forceinline__ void mma_issue(uint32_t d_tmem, uint64_t adesc, uint6
             : "memory");
 }
 
-// The same two instructions for a converged warp: every lane executes them, lane 0's predicate lets
-// them through (no branch).  Descriptors are passed as their low words; the high word is constant.
+// The same two instructions for a converged warp: every lane executes them and the predicate lets
+// one through (`on` is non-zero in lane 0 only, and only if the step is to be issued), so there
+// is no branch.  Descriptors are passed as their low words; the high word is constant.
 constexpr uint32_t kDescHi = (256u >> 4) | (1u << 14);   // stride byte offset 256, descriptor version 1
 template <bool I8>
-__device__ __forceinline__ void mma_issue_lane0(int lane, uint32_t d_tmem, uint32_t adesc_lo, uint32_t bdesc_lo,
-                                                uint32_t accumulate) {
+__device__ __forceinline__ void mma_issue_if(uint32_t on, uint32_t d_tmem, uint32_t adesc_lo, uint32_t bdesc_lo,
+                                             uint32_t accumulate) {
     if (I8)
         asm volatile(
             "{\n\t.reg .pred p, q;\n\t.reg .b64 da, db;\n\t"
-            "setp.ne.b32 p, %4, 0;\n\tsetp.eq.s32 q, %5, 0;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\tsetp.ne.b32 q, %5, 0;\n\t"
             "mov.b64 da, {%1, %6};\n\tmov.b64 db, {%2, %6};\n\t"
             "@q tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %3, p;\n\t}"
-            ::"r"(d_tmem), "r"(adesc_lo), "r"(bdesc_lo), "r"(kIdescI8), "r"(accumulate), "r"(lane), "r"(kDescHi)
+            ::"r"(d_tmem), "r"(adesc_lo), "r"(bdesc_lo), "r"(kIdescI8), "r"(accumulate), "r"(on), "r"(kDescHi)
             : "memory");
     else
         asm volatile(
             "{\n\t.reg .pred p, q;\n\t.reg .b64 da, db;\n\t"
-            "setp.ne.b32 p, %4, 0;\n\tsetp.eq.s32 q, %5, 0;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\tsetp.ne.b32 q, %5, 0;\n\t"
             "mov.b64 da, {%1, %6};\n\tmov.b64 db, {%2, %6};\n\t"
             "@q tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], da, db, %3, p;\n\t}"
-            ::"r"(d_tmem), "r"(adesc_lo), "r"(bdesc_lo), "r"(kIdescF8), "r"(accumulate), "r"(lane), "r"(kDescHi)
+            ::"r"(d_tmem), "r"(adesc_lo), "r"(bdesc_lo), "r"(kIdescF8), "r"(accumulate), "r"(on), "r"(kDescHi)
             : "memory");
 }
-__device__ __forceinline__ void mma_commit_lane0(int lane, uint32_t bar_s) {
+__device__ __forceinline__ void mma_commit_if(uint32_t on, uint32_t bar_s) {
     asm volatile(
-        "{\n\t.reg .pred q;\n\tsetp.eq.s32 q, %1, 0;\n\t"
+        "{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
         "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
-        ::"r"(bar_s), "r"(lane)
+        ::"r"(bar_s), "r"(on)
         : "memory");
 }
 // low word of the operand descriptor of a block at shared address saddr (leading byte offset 128)
@@ -522,23 +523,34 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
             // independent and two warps take them in turn (even and odd slots), so that each has two
             // groups' time for its bookkeeping; wider groups chain into one slot and stay with one warp.
             const uint32_t me = (uint32_t)(warp - kMmaWarp);
+            const uint32_t lane0 = lane == 0 ? 1u : 0u;
             const uint32_t ares_lo = desc_lo(ares_s), ring_lo = desc_lo(ring_s);
             const uint32_t stage_step = a.stage_bytes >> 4, n_stages = (uint32_t)a.n_stages;
             const uint32_t a_in_stage = resident ? 0u : (uint32_t)(kChunk * (kBlock >> 4));
             const uint32_t empty_s = smem_u32(&c->empty[0]), tfull_s = smem_u32(&c->tfull[0]);
             const uint32_t tempty_s = smem_u32(&c->tempty[0]);
             const int n_steps = a.n_steps;
+            // Group k of a tile uses TMEM slot k & 3, so a chunk of four steps always starts at slot 0.
             auto role = [&](auto dual_tag) {
                 constexpr bool DUAL = decltype(dual_tag)::value;
-                uint32_t s = 0, ph = 0, slot = 0, tph = 0, ic = 0;
-                bool slot_ready = false;   // the early answer about this warp's next slot, if it was yes
+                uint32_t s = 0, ph = 0, ic = 0;
                 bool ok = true;
+                // DUAL: this warp's two slots (me and me + 2), everything about them precomputed
+                const uint32_t tm_a = tmem_base + me * kBN, tm_b = tm_a + 2 * kBN;
+                const uint32_t off_a = me * (kBlock >> 4), off_b = off_a + 2 * (kBlock >> 4);
+                const uint32_t tfull_a = tfull_s + me * 8, tfull_b = tfull_a + 16;
+                const uint32_t tempty_a = tempty_s + me * 8, tempty_b = tempty_a + 16;
+                uint32_t q_a = 1, q_b = 1;     // parity to wait for on tempty of each slot; a fresh barrier passes parity 1
+                // otherwise: one slot at a time
+                uint32_t qm = 0xFu;            // the same parities as a mask, bit = slot
                 for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++ic) {
                     const int part = item % a.n_parts;
                     const int n_tiles = part_begin(part + 1) - part_begin(part);
                     ok = mbar_wait_warp(&c->a_full, ic & 1, c, a.status, 6u);
                     for (int tl = 0; tl < n_tiles && ok; ++tl) {
                         int sub = 0;
+                        uint32_t slot = 0;
+                        bool slot_ready = false;   // the early answer about the next slot, if it was yes
                         uint32_t a_lo = ares_lo;   // resident: walks through the item's A blocks
                         for (int k0 = 0; k0 < n_steps && ok; k0 += kChunk) {
                             ok = mbar_wait_warp(&c->full[s], ph, c, a.status, 4u);
@@ -546,50 +558,53 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
                             const uint32_t b_lo = ring_lo + s * stage_step;
                             if (!resident) a_lo = b_lo + a_in_stage;
                             const int nk = min(kChunk, n_steps - k0);
-#pragma unroll
-                            for (int j = 0; j < kChunk; ++j) {
-                                if (j < nk) {
-                                    if (DUAL) {
-                                        if ((slot & 1u) == me) {
-                                            if (!slot_ready) {
-                                                ok = mbar_wait_warp(&c->tempty[slot], tph ^ 1, c, a.status, 3u);
-                                                if (!ok) break;
-                                            }
-                                            // ask about this warp's next slot now: the answer travels while this step is issued
-                                            slot_ready = __all_sync(0xffffffffu, mbar_test_s(tempty_s + (slot ^ 2u) * 8,
-                                                                                             tph ^ (slot >> 1) ^ 1u));
-                                            tc_fence_after();
-                                            mma_issue_lane0<I8>(lane, tmem_base + slot * kBN, a_lo + j * (kBlock >> 4),
-                                                                b_lo + j * (kBlock >> 4), 0u);
-                                            mma_commit_lane0(lane, tfull_s + slot * 8);
-                                        }
+                            if (DUAL) {
+                                // straight-line: both of this warp's steps, predicated off past the end of K
+                                const uint32_t act_a = me < (uint32_t)nk ? 1u : 0u, act_b = me + 2 < (uint32_t)nk ? 1u : 0u;
+                                const bool rdy_a = mbar_test_s(tempty_a, q_a) || !act_a;
+                                const bool rdy_b = mbar_test_s(tempty_b, q_b) || !act_b;
+                                if (!__all_sync(0xffffffffu, rdy_a)) {
+                                    ok = mbar_wait_warp(&c->tempty[me], q_a, c, a.status, 3u);
+                                    if (!ok) break;
+                                }
+                                tc_fence_after();
+                                mma_issue_if<I8>(lane0 & act_a, tm_a, a_lo + off_a, b_lo + off_a, 0u);
+                                mma_commit_if(lane0 & act_a, tfull_a);
+                                q_a ^= act_a;
+                                if (!__all_sync(0xffffffffu, rdy_b)) {
+                                    ok = mbar_wait_warp(&c->tempty[me + 2], q_b, c, a.status, 3u);
+                                    if (!ok) break;
+                                    tc_fence_after();
+                                }
+                                mma_issue_if<I8>(lane0 & act_b, tm_b, a_lo + off_b, b_lo + off_b, 0u);
+                                mma_commit_if(lane0 & act_b, tfull_b);
+                                q_b ^= act_b;
+                            } else {
+                                uint32_t a_j = a_lo, b_j = b_lo;
+#pragma unroll 1
+                                for (int j = 0; j < nk; ++j, a_j += kBlock >> 4, b_j += kBlock >> 4) {
+                                    if (sub == 0 && !slot_ready) {
+                                        ok = mbar_wait_warp(&c->tempty[slot], (qm >> slot) & 1u, c, a.status, 3u);
+                                        if (!ok) break;
+                                    }
+                                    tc_fence_after();
+                                    mma_issue_if<I8>(lane0, tmem_base + slot * kBN, a_j, b_j, sub == 0 ? 0u : 1u);
+                                    if (++sub == spg) {
+                                        sub = 0;
+                                        mma_commit_if(lane0, tfull_s + slot * 8);
+                                        qm ^= 1u << slot;
                                         slot = (slot + 1) & (kSlots - 1);
-                                        tph ^= (slot == 0);
-                                    } else {
-                                        if (sub == 0 && !slot_ready) {
-                                            ok = mbar_wait_warp(&c->tempty[slot], tph ^ 1, c, a.status, 3u);
-                                            if (!ok) break;
-                                        }
-                                        tc_fence_after();
-                                        mma_issue_lane0<I8>(lane, tmem_base + slot * kBN, a_lo + j * (kBlock >> 4),
-                                                            b_lo + j * (kBlock >> 4), sub == 0 ? 0u : 1u);
-                                        if (++sub == spg) {
-                                            sub = 0;
-                                            mma_commit_lane0(lane, tfull_s + slot * 8);
-                                            slot = (slot + 1) & (kSlots - 1);
-                                            tph ^= (slot == 0);
-                                            slot_ready = __all_sync(0xffffffffu, mbar_test_s(tempty_s + slot * 8, tph ^ 1u));
-                                        }
+                                        slot_ready = __all_sync(0xffffffffu, mbar_test_s(tempty_s + slot * 8, (qm >> slot) & 1u));
                                     }
                                 }
+                                if (!ok) break;
                             }
-                            if (!ok) break;
                             if (resident) a_lo += kChunk * (kBlock >> 4);
-                            mma_commit_lane0(lane, empty_s + s * 8);
+                            mma_commit_if(lane0, empty_s + s * 8);
                             if (++s == n_stages) { s = 0; ph ^= 1; }
                         }
                     }
-                    if (ok) mma_commit_lane0(lane, smem_u32(&c->a_empty));
+                    if (ok) mma_commit_if(lane0, smem_u32(&c->a_empty));
                 }
             };
             if (spg == 1) role(std::true_type{});
@@ -619,20 +634,13 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
         const uint32_t my_scale_s = scales_s + (uint32_t)row * 4;
         const size_t row_step = (size_t)kRPI * (size_t)a.y_stride * esz;
 
-        // groups this CTA will see, so that the next slot can be requested early
-        uint32_t total = 0;
-        for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
-            const int part = item % a.n_parts;
-            total += (uint32_t)(part_begin(part + 1) - part_begin(part)) * (uint32_t)a.Kg;
-        }
-
         uint64_t yacc[kCols / 2];      // 32 floats of one output row, packed in pairs
         uint32_t v[kCols];             // landing buffer: this thread's 32 columns of a slot
 #pragma unroll
         for (int q = 0; q < kCols; ++q) v[q] = 0u;
-        uint32_t gc = 0, slot = 0, tph = 0, ic = 0;   // groups, their slot and phase; items so far
-        int item = blockIdx.x, mt = 0, nt = 0, nt_end = 0, grp_left = 0;
-        uint32_t scale_s = my_scale_s;   // this row's scale of the group about to be promoted
+        uint32_t ic = 0;                 // items so far
+        uint32_t p_full[kSlots] = {0u, 0u, 0u, 0u};   // parity of the completion of tfull[s] to wait for next
+        int item = blockIdx.x, mt = 0, nt = 0, nt_end = 0;
         int64_t m = 0, n0 = 0;
         int rows_left = 0;               // rows of y from this lane's first output row to the end
         float ws[kCPL], bs[kCPL];        // s_o * 2^e and bias of the columns this lane writes
@@ -651,8 +659,6 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
         };
         auto begin_tile = [&]() {
             n0 = (int64_t)nt * kBN + col0;
-            grp_left = a.Kg;
-            scale_s = my_scale_s;
 #pragma unroll
             for (int j = 0; j < kCols / 2; ++j) yacc[j] = 0ull;
             // vector stores: this lane writes columns n0 + cl * kCPL ...; otherwise column n0 + lane
@@ -737,26 +743,30 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
             }
             if (ok && item < n_items) begin_tile();
         };
-        // One group: its 32 columns were requested earlier and land in v.  Release the slot as soon as
-        // they have landed, fold them in, then request the next group (after the epilogue at the end
-        // of a tile: the next group may belong to the next work item, which cannot start before this
-        // warp has handed the current item's buffers back).  With four promotion warps per scheduler
-        // the load of one warp hides behind the FMAs of the others.
+        // Group k of a tile lives in TMEM slot k & 3, so the slot is a compile-time constant in a loop
+        // unrolled by four.  request<U>: wait until slot U is full, start loading this thread's 32
+        // columns into v.  consume<U>: wait for them, hand the slot back at once, fold them in; it also
+        // asks whether the next slot is full already, an answer that is only needed after the FMAs.
+        // With four promotion warps per scheduler the load of one warp hides behind the FMAs of the others.
         const uint32_t tfull_s = smem_u32(&c->tfull[0]), tempty_s = smem_u32(&c->tempty[0]);
-        auto promote = [&]() {
-            const uint32_t dbits = lds32(scale_s);
-            scale_s += kScaleBlock;
+        auto request = [&](auto u_tag, bool ready) {
+            constexpr uint32_t U = decltype(u_tag)::value;
+            if (!__all_sync(0xffffffffu, ready)) ok = mbar_wait_warp(&c->tfull[U], p_full[U], c, a.status, 2u);
+            p_full[U] ^= 1u;
+            tc_fence_after();
+            tmem_ld32(tmem_row + U * kBN, v);
+        };
+        auto consume = [&](auto u_tag, uint32_t scale_q, int k) -> bool {
+            constexpr uint32_t U = decltype(u_tag)::value, N = (U + 1) & (kSlots - 1);
+            const uint32_t dbits = lds32(scale_q + U * kScaleBlock);
             const uint64_t d2 = pack2(dbits, dbits);
-            // ask about the next group's slot now; the answer is needed only after the FMAs below
-            const uint32_t nslot = (slot + 1) & (kSlots - 1), ntph = tph ^ (nslot == 0);
-            const bool more = gc + 1 < total;
-            const bool next_ready = mbar_test_s(tfull_s + nslot * 8, ntph) || !more;
+            const bool next_ready = mbar_test_s(tfull_s + N * 8, p_full[N]);
             tmem_ld_wait();                               // v has landed: the slot is drained
             tc_fence_before();
             __syncwarp();
-            mbar_arrive_lane0_s(tempty_s + slot * 8, lane);
+            mbar_arrive_lane0_s(tempty_s + U * 8, lane);
             if (DBG) {
-                if (a.acc_debug && row_ok) debug_store<I8>(a, v, m, n0, a.Kg - grp_left);
+                if (a.acc_debug && row_ok) debug_store<I8>(a, v, m, n0, k + (int)U);
             }
             if (I8) {
 #pragma unroll
@@ -764,30 +774,53 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
             }
 #pragma unroll
             for (int q = 0; q < kCols / 2; ++q) fma2(yacc[q], pack2(v[2 * q], v[2 * q + 1]), d2);
-            slot = nslot;
-            tph = ntph;
-            ++gc;
-            if (--grp_left == 0) {
-                finish_tile();
-                if (!ok || !more) return;
-                ok = mbar_wait_warp(&c->tfull[slot], tph, c, a.status, 2u);
-            } else if (!__all_sync(0xffffffffu, next_ready)) {
-                ok = mbar_wait_warp(&c->tfull[slot], tph, c, a.status, 2u);
-            }
-            tc_fence_after();
-            tmem_ld32(tmem_row + slot * kBN, v);
+            return next_ready;
         };
+        const std::integral_constant<uint32_t, 0> u0{};
+        const std::integral_constant<uint32_t, 1> u1{};
+        const std::integral_constant<uint32_t, 2> u2{};
+        const std::integral_constant<uint32_t, 3> u3{};
 
-        if (total > 0) {
+        if (item < n_items) {
             begin_item();
             if (ok) {
                 begin_tile();
-                ok = mbar_wait_warp(&c->tfull[0], 0, c, a.status, 2u);
+                request(u0, false);
             }
-            tc_fence_after();
-            tmem_ld32(tmem_row, v);
 #pragma unroll 1
-            while (ok && gc < total) promote();
+            while (ok && item < n_items) {
+                // one tile; the load of its first group is in flight
+                const int Kg = a.Kg;
+                uint32_t scale_q = my_scale_s;
+                int k = 0;
+#pragma unroll 1
+                for (; k + 4 < Kg && ok; k += 4, scale_q += 4 * kScaleBlock) {   // four groups, and more behind them
+                    request(u1, consume(u0, scale_q, k));
+                    request(u2, consume(u1, scale_q, k));
+                    request(u3, consume(u2, scale_q, k));
+                    request(u0, consume(u3, scale_q, k));
+                }
+                if (!ok) break;
+                const int rem = Kg - k;                   // the last one to four groups
+                bool r = consume(u0, scale_q, k);
+                if (rem > 1) {
+                    request(u1, r);
+                    r = consume(u1, scale_q, k);
+                    if (rem > 2) {
+                        request(u2, r);
+                        r = consume(u2, scale_q, k);
+                        if (rem > 3) {
+                            request(u3, r);
+                            consume(u3, scale_q, k);
+                        }
+                    }
+                }
+                if (!ok) break;
+                // The epilogue comes before the wait for the next tile's first group: that group may belong
+                // to the next work item, which cannot start before this warp has handed the item's buffers back.
+                finish_tile();
+                if (ok && item < n_items) request(u0, false);
+            }
         }
         tmem_ld_wait();            // nothing may still be landing when TMEM is released
     }
