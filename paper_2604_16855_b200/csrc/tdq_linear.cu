@@ -48,6 +48,7 @@
 // Every wait on an mbarrier is bounded: after about a second the thread records a code in the
 // workspace status word and raises a CTA-wide flag; every role then leaves its loops, the CTA
 // releases its TMEM and returns.
+#include <cuda.h>
 #include <mutex>
 #include <type_traits>
 
@@ -71,6 +72,7 @@ constexpr int kCols = kBN / (kPromoWarps / 4);   // 32 columns of one row per pr
 constexpr int kThreads = (kPromoWarp0 + kPromoWarps) * 32;   // 640
 constexpr int kStripBytes = kCols * 4;   // one thread's 32 raw fp32 sums
 constexpr int kStagingBytes = kPromoWarps * 32 * kStripBytes;
+constexpr int kWsbBytes = kPromoWarps * 256;   // per warp: 32 output-channel scales and 32 biases
 constexpr int kCtrlBytes = 256;
 constexpr int kSmemLimit = 232448;       // 227 KB per CTA
 constexpr uint32_t kTmemCols = kSlots * kBN;
@@ -101,7 +103,7 @@ struct LinArgs {
     int64_t y_stride;
     int32_t* acc_debug;
     uint32_t* status;
-    int32_t vec_ok;            // y rows can be written with 16-byte aligned vector stores
+    int32_t tma_ok;            // y can be written with bulk tensor stores (16-byte aligned base and row pitch)
     float out_scale;           // 2^18 (E4M3 route) or 2^-8 (int8 route)
 };
 
@@ -342,6 +344,21 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint32_t x, uint32_t y, ui
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
 }
 
+// shared -> global bulk tensor store of one box (coordinates: column, row), tracked by bulk groups
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src_smem, int32_t x, int32_t y) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src_smem), "r"(x), "r"(y)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_group_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_group0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ uint32_t lds16(uint32_t addr) {
+    uint16_t v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr) : "memory");
+    return v;
+}
+
 template <int N>
 __device__ __forceinline__ void setmaxnreg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N>
@@ -430,7 +447,7 @@ __device__ __noinline__ void debug_store(const LinArgs& a, const uint32_t* v, in
 }
 
 template <bool I8, bool YBF16, bool DBG>
-__global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
+__global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a, const __grid_constant__ CUtensorMap ymap) {
     extern __shared__ __align__(128) uint8_t smem_raw[];   // no static shared memory: the window starts aligned
     Ctrl* c = reinterpret_cast<Ctrl*>(smem_raw);
     const uint32_t sm_s = smem_u32(smem_raw);
@@ -619,20 +636,19 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
         const int col0 = (pw >> 2) * kCols;
         const uint32_t tmem_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + col0;
         // Epilogue geometry.  A warp owns one 32 x 32 block of every tile (the rows of its TMEM lanes,
-        // its 32 columns) and needs no other warp to write it out: it parks the raw sums in 4 KB of
-        // shared memory of its own, one 128-byte row per lane, and reads them back with kLPR lanes per
-        // row, so that a store instruction writes whole 128-byte (fp32) or 64-byte (bf16) row segments.
-        // On the way back a lane always meets the same columns and keeps their scales in registers.
+        // its 32 columns) and needs no other warp to write it out: it scales the sums, parks them in
+        // 4 KB of shared memory of its own in the layout of a bulk tensor store (rows of 128 or 64
+        // bytes, 16-byte chunks swizzled by the row so that the writes are conflict-free), and lane 0
+        // starts the store.  The copy engine clips the box at the edges of y and runs while the warp
+        // promotes the next tile; the strip is reused only after the engine has read it.
         constexpr int esz = YBF16 ? 2 : 4;
-        constexpr int kLPR = YBF16 ? 4 : 8;           // lanes per row on the way out
-        constexpr int kRPI = 32 / kLPR;               // rows per store instruction
-        constexpr int kCPL = kCols / kLPR;            // columns per lane: 16 bytes of y
-        const int sub = lane / kLPR, cl = lane % kLPR;
-        const uint32_t strip_w = sm_s + a.staging_off + (uint32_t)pw * (32 * kStripBytes);
-        // 16-byte chunk j of row r sits at chunk position j ^ (r & 7): conflict-free both ways
-        const uint32_t strip_wr = (strip_w + (uint32_t)lane * kStripBytes) ^ (((uint32_t)lane & 7u) << 4);
+        constexpr uint32_t kRowBytes = kCols * esz;   // one row of the strip
+        const uint32_t strips_s = (sm_s + a.staging_off + 1023u) & ~1023u;   // the swizzle pattern repeats every 1024 bytes
+        const uint32_t strip_w = strips_s + (uint32_t)pw * (32 * kStripBytes);
+        const uint32_t strip_row = strip_w + (uint32_t)lane * kRowBytes;
+        const uint32_t swz = YBF16 ? (((uint32_t)lane >> 1) & 3u) : ((uint32_t)lane & 7u);   // chunk c sits at c ^ swz
+        const uint32_t wsb_s = strips_s + kStagingBytes + (uint32_t)pw * 256;
         const uint32_t my_scale_s = scales_s + (uint32_t)row * 4;
-        const size_t row_step = (size_t)kRPI * (size_t)a.y_stride * esz;
 
         uint64_t yacc[kCols / 2];      // 32 floats of one output row, packed in pairs
         uint32_t v[kCols];             // landing buffer: this thread's 32 columns of a slot
@@ -642,9 +658,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
         uint32_t p_full[kSlots] = {0u, 0u, 0u, 0u};   // parity of the completion of tfull[s] to wait for next
         int item = blockIdx.x, mt = 0, nt = 0, nt_end = 0;
         int64_t m = 0, n0 = 0;
-        int rows_left = 0;               // rows of y from this lane's first output row to the end
-        float ws[kCPL], bs[kCPL];        // s_o * 2^e and bias of the columns this lane writes
-        bool ok = true, row_ok = false, col_ok = false;
+        float w0 = 0.f, b0 = 0.f;        // channel scale and bias of column n0 + lane
+        bool ok = true, row_ok = false;
 
         auto begin_item = [&]() {
             mt = item / a.n_parts;
@@ -653,83 +668,71 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
             nt_end = part_begin(part + 1);
             m = (int64_t)mt * kBM + row;
             row_ok = m < a.M;
-            const int64_t m_out = (int64_t)mt * kBM + quarter * 32 + (a.vec_ok ? sub : 0);
-            rows_left = (int)min((int64_t)32, max((int64_t)0, a.M - m_out));
             ok = mbar_wait_warp(&c->a_full, ic & 1, c, a.status, 7u);
         };
         auto begin_tile = [&]() {
             n0 = (int64_t)nt * kBN + col0;
 #pragma unroll
             for (int j = 0; j < kCols / 2; ++j) yacc[j] = 0ull;
-            // vector stores: this lane writes columns n0 + cl * kCPL ...; otherwise column n0 + lane
-            const int64_t cb = n0 + (a.vec_ok ? cl * kCPL : lane);
-            col_ok = cb < a.O;
-#pragma unroll
-            for (int e = 0; e < kCPL; ++e) {
-                const bool in = cb + e < a.O && (a.vec_ok || e == 0);
-                ws[e] = in ? __fmul_rn(__ldg(a.wscale + cb + e), a.out_scale) : 0.f;
-                bs[e] = (in && a.bias) ? __ldg(a.bias + cb + e) : 0.f;
-            }
+            // loaded now, used at the end of the tile: the latency is not waited for
+            const int64_t ca = n0 + lane;
+            w0 = ca < a.O ? __ldg(a.wscale + ca) : 0.f;
+            b0 = (a.bias && ca < a.O) ? __ldg(a.bias + ca) : 0.f;
         };
         // y = (s_o * 2^e) * sum + bias for the tile that just finished, then on to the next tile
         auto finish_tile = [&]() {
+            if (lane == 0) bulk_wait_group_read0();      // the previous tile's store has read the strip
+            sts32(wsb_s + lane * 4, __float_as_uint(__fmul_rn(w0, a.out_scale)));
+            sts32(wsb_s + 128 + lane * 4, __float_as_uint(b0));
+            __syncwarp();
 #pragma unroll
             for (int j = 0; j < kCols / 4; ++j) {
                 float o0, o1, o2, o3;
                 unpack2(yacc[2 * j], o0, o1);
                 unpack2(yacc[2 * j + 1], o2, o3);
-                sts128(strip_wr ^ ((uint32_t)j << 4), __float_as_uint(o0), __float_as_uint(o1), __float_as_uint(o2),
-                       __float_as_uint(o3));
+                const uint4 s4 = lds128(wsb_s + j * 16), b4 = lds128(wsb_s + 128 + j * 16);
+                o0 = __fmaf_rn(__uint_as_float(s4.x), o0, __uint_as_float(b4.x));
+                o1 = __fmaf_rn(__uint_as_float(s4.y), o1, __uint_as_float(b4.y));
+                o2 = __fmaf_rn(__uint_as_float(s4.z), o2, __uint_as_float(b4.z));
+                o3 = __fmaf_rn(__uint_as_float(s4.w), o3, __uint_as_float(b4.w));
+                if (YBF16) {       // columns 4 j .. 4 j + 3: half of chunk j / 2
+                    __nv_bfloat162 lo = __floats2bfloat162_rn(o0, o1);
+                    __nv_bfloat162 hi = __floats2bfloat162_rn(o2, o3);
+                    sts64(strip_row + ((((uint32_t)j >> 1) ^ swz) << 4) + ((uint32_t)j & 1u) * 8,
+                          *reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+                } else {
+                    sts128(strip_row + (((uint32_t)j ^ swz) << 4), __float_as_uint(o0), __float_as_uint(o1),
+                           __float_as_uint(o2), __float_as_uint(o3));
+                }
             }
-            __syncwarp();
-            if (a.vec_ok) {
-                uint8_t* dst = reinterpret_cast<uint8_t*>(a.y) +
-                               ((size_t)((int64_t)mt * kBM + quarter * 32 + sub) * a.y_stride + (size_t)(n0 + cl * kCPL)) * esz;
-#pragma unroll
-                for (int it = 0; it < kLPR; ++it) {
-                    const uint32_t r = (uint32_t)(it * kRPI + sub);
-                    float o[kCPL];
-#pragma unroll
-                    for (int e4 = 0; e4 < kCPL / 4; ++e4) {
-                        const uint32_t ch = (uint32_t)(cl * (kCPL / 4) + e4);
-                        const uint4 q = lds128(strip_w + r * kStripBytes + ((ch ^ (r & 7u)) << 4));
-                        o[4 * e4 + 0] = __fmaf_rn(ws[4 * e4 + 0], __uint_as_float(q.x), bs[4 * e4 + 0]);
-                        o[4 * e4 + 1] = __fmaf_rn(ws[4 * e4 + 1], __uint_as_float(q.y), bs[4 * e4 + 1]);
-                        o[4 * e4 + 2] = __fmaf_rn(ws[4 * e4 + 2], __uint_as_float(q.z), bs[4 * e4 + 2]);
-                        o[4 * e4 + 3] = __fmaf_rn(ws[4 * e4 + 3], __uint_as_float(q.w), bs[4 * e4 + 3]);
-                    }
-                    if (it * kRPI < rows_left && col_ok) {
-                        uint4 val;
-                        if (YBF16) {
-                            __nv_bfloat162 h0 = __floats2bfloat162_rn(o[0], o[1]);
-                            __nv_bfloat162 h1 = __floats2bfloat162_rn(o[2], o[3]);
-                            __nv_bfloat162 h2 = __floats2bfloat162_rn(o[kCPL - 4], o[kCPL - 3]);
-                            __nv_bfloat162 h3 = __floats2bfloat162_rn(o[kCPL - 2], o[kCPL - 1]);
-                            val = make_uint4(*reinterpret_cast<uint32_t*>(&h0), *reinterpret_cast<uint32_t*>(&h1),
-                                             *reinterpret_cast<uint32_t*>(&h2), *reinterpret_cast<uint32_t*>(&h3));
-                        } else {
-                            val = make_uint4(__float_as_uint(o[0]), __float_as_uint(o[1]), __float_as_uint(o[2]),
-                                             __float_as_uint(o[3]));
-                        }
-                        __stcs(reinterpret_cast<uint4*>(dst + (size_t)it * row_step), val);
-                    }
+            const int64_t m0 = (int64_t)mt * kBM + quarter * 32;   // first row of this warp's block
+            if (a.tma_ok) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes before the engine's reads
+                __syncwarp();
+                if (lane == 0 && m0 < a.M && n0 < a.O) {
+                    tma_store_2d(&ymap, strip_w, (int32_t)n0, (int32_t)m0);
+                    bulk_commit_group();
                 }
             } else {          // any alignment: a row at a time, lane = column
+                __syncwarp();
+                const int rows = (int)min((int64_t)32, a.M - m0);
+                if (n0 + lane < a.O) {
 #pragma unroll 1
-                for (int r = 0; r < rows_left; ++r) {
-                    const uint32_t word = lds32(strip_w + (uint32_t)r * kStripBytes +
-                                                ((((uint32_t)lane >> 2) ^ ((uint32_t)r & 7u)) << 4) + ((uint32_t)lane & 3u) * 4);
-                    const float o = __fmaf_rn(ws[0], __uint_as_float(word), bs[0]);
-                    const int64_t mg = (int64_t)mt * kBM + quarter * 32 + r;
-                    if (col_ok) {
-                        if (YBF16)
-                            reinterpret_cast<__nv_bfloat16*>(a.y)[mg * a.y_stride + n0 + lane] = __float2bfloat16_rn(o);
-                        else
-                            reinterpret_cast<float*>(a.y)[mg * a.y_stride + n0 + lane] = o;
+                    for (int r = 0; r < rows; ++r) {
+                        const size_t at = (size_t)(m0 + r) * a.y_stride + (size_t)(n0 + lane);
+                        if (YBF16) {
+                            const uint32_t rs = ((uint32_t)r >> 1) & 3u;
+                            reinterpret_cast<uint16_t*>(a.y)[at] = (uint16_t)lds16(
+                                strip_w + (uint32_t)r * kRowBytes + ((((uint32_t)lane >> 3) ^ rs) << 4) + ((uint32_t)lane & 7u) * 2);
+                        } else {
+                            const uint32_t rs = (uint32_t)r & 7u;
+                            reinterpret_cast<uint32_t*>(a.y)[at] = lds32(
+                                strip_w + (uint32_t)r * kRowBytes + ((((uint32_t)lane >> 2) ^ rs) << 4) + ((uint32_t)lane & 3u) * 4);
+                        }
                     }
                 }
+                __syncwarp();     // the strip may be overwritten by the next tile
             }
-            __syncwarp();     // the strip may be overwritten by the next tile
             // next tile, next item
             if (++nt == nt_end) {
                 // the item's scales were read through the generic proxy; the next item's bulk copies
@@ -823,6 +826,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
             }
         }
         tmem_ld_wait();            // nothing may still be landing when TMEM is released
+        if (lane == 0) bulk_wait_group0();   // nor may a store still be reading this CTA's shared memory
     }
 
     tc_fence_before();
@@ -838,6 +842,33 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(LinArgs a) {
 
 // ------------------------------------------------------------------------------------------
 // host side
+
+// Descriptor of y for the epilogue's bulk tensor stores: a [M][O] matrix with a row pitch, written in
+// boxes of 32 rows x 32 columns whose 16-byte chunks are swizzled in shared memory the way the
+// kernel lays them out (128-byte rows: chunk ^ (row & 7); 64-byte rows: chunk ^ ((row >> 1) & 3)).
+// The driver's encoder is looked up once; false when it is not there or refuses the shape.
+typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                      const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                      CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+bool encode_y_map(CUtensorMap* map, void* y, bool bf16, int64_t M, int64_t O, int64_t y_row_stride) {
+    static const TensorMapEncodeFn encode = [] {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult res;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &res) != cudaSuccess ||
+            res != cudaDriverEntryPointSuccess)
+            fn = nullptr;
+        return reinterpret_cast<TensorMapEncodeFn>(fn);
+    }();
+    if (!encode) return false;
+    const cuuint64_t esz = bf16 ? 2 : 4;
+    const cuuint64_t dims[2] = {(cuuint64_t)O, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)y_row_stride * esz};
+    const cuuint32_t box[2] = {(cuuint32_t)kCols, 32u};
+    const cuuint32_t elem_strides[2] = {1u, 1u};
+    return encode(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, y, dims, strides, box,
+                  elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, bf16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
 
 struct Plan {
     int64_t tiles_m, tiles_n;
@@ -861,7 +892,7 @@ bool make_plan(int64_t M, int64_t I_pad, int64_t O, int32_t g, int n_sm, Plan& p
     p.s_bytes = (size_t)p.tiles_m * p.Kg * kScaleBlock;
     // shared memory: control, the item's scales, [resident A], ring, output strips, channel scales
     const int64_t scales = (int64_t)p.Kg * kScaleBlock;
-    const int64_t fixed = 128 + kCtrlBytes + scales + kStagingBytes;
+    const int64_t fixed = 1024 + kCtrlBytes + scales + kStagingBytes + kWsbBytes;   // 1024: the strips start on a 1 KB boundary
     const int64_t a_res = (int64_t)p.n_steps * kBlock;
     const int64_t stage_b = (int64_t)kChunk * kBlock, stage_ab = 2 * stage_b;
     const int64_t stages_res = (kSmemLimit - fixed - a_res) / stage_b;
@@ -880,7 +911,7 @@ bool make_plan(int64_t M, int64_t I_pad, int64_t O, int32_t g, int n_sm, Plan& p
         p.ring_off = p.ares_off;
     }
     p.staging_off = p.ring_off + (uint32_t)p.n_stages * p.stage_bytes;
-    p.smem_bytes = p.staging_off + kStagingBytes + 128;
+    p.smem_bytes = p.staging_off + 1024 + kStagingBytes + kWsbBytes;
     // split the column tiles of a row block into parts so that the items fill the SMs evenly
     int best = 1;
     int64_t best_cost = INT64_MAX;
@@ -968,12 +999,17 @@ extern "C" tdq_status tdq_w4a4_linear(const uint8_t* xcodes, const float* xscale
     a.y = y; a.y_stride = y_row_stride; a.acc_debug = acc_debug;
     a.status = reinterpret_cast<uint32_t*>(workspace);
     const int64_t esz = y_dtype == TDQ_BF16 ? 2 : 4;
-    // vector stores: every 16-byte chunk of a tile row is aligned and lies wholly inside or outside y
-    a.vec_ok = (reinterpret_cast<uintptr_t>(y) % 16 == 0 && (y_row_stride * esz) % 16 == 0 && (O * esz) % 16 == 0) ? 1 : 0;
+    // bulk tensor stores want a 16-byte aligned base and row pitch; anything else goes element by element
+    CUtensorMap ymap;
+    memset(&ymap, 0, sizeof(ymap));
+    a.tma_ok = 0;
+    if (reinterpret_cast<uintptr_t>(y) % 16 == 0 && (y_row_stride * esz) % 16 == 0 && O <= INT32_MAX && M <= INT32_MAX &&
+        encode_y_map(&ymap, y, y_dtype == TDQ_BF16, M, O, y_row_stride))
+        a.tma_ok = 1;
     a.out_scale = i8 ? 0.00390625f : 262144.0f;
 
     const bool ybf = y_dtype == TDQ_BF16, dbg = acc_debug != nullptr;
-    void (*kernel)(LinArgs) = nullptr;
+    void (*kernel)(LinArgs, CUtensorMap) = nullptr;
 #define TDQ_PICK(I8_, YB_, DBG_) if (i8 == I8_ && ybf == YB_ && dbg == DBG_) kernel = w4a4_gemm_kernel<I8_, YB_, DBG_>;
     TDQ_PICK(false, false, false) TDQ_PICK(false, true, false) TDQ_PICK(true, false, false) TDQ_PICK(true, true, false)
     TDQ_PICK(false, false, true) TDQ_PICK(false, true, true) TDQ_PICK(true, false, true) TDQ_PICK(true, true, true)
@@ -992,7 +1028,7 @@ extern "C" tdq_status tdq_w4a4_linear(const uint8_t* xcodes, const float* xscale
 
     const int64_t items = p.tiles_m * p.n_parts;
     const unsigned grid = (unsigned)(items < n_sm ? items : n_sm);
-    kernel<<<grid, kThreads, p.smem_bytes, stream>>>(a);
+    kernel<<<grid, kThreads, p.smem_bytes, stream>>>(a, ymap);
     if (cudaGetLastError() != cudaSuccess) return TDQ_ERR_CUDA;
     g_launch_count.fetch_add(1, std::memory_order_relaxed);
     return TDQ_OK;
