@@ -77,6 +77,7 @@ constexpr int kCtrlBytes = 256;
 constexpr int kSmemLimit = 232448;       // 227 KB per CTA
 constexpr uint32_t kTmemCols = kSlots * kBN;
 constexpr long long kTimeoutCycles = 2000000000LL;
+constexpr uint32_t kSuspendHintNs = 20000;   // longest sleep of one try_wait
 constexpr int kExpandThreads = 512;
 constexpr int kRegsControl = 40, kRegsPromo = 104;   // 128 * 40 + 512 * 104 <= 640 * 96
 
@@ -139,35 +140,31 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
 }
 
 __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;   // try_wait may suspend the thread for a short, hardware-chosen time before it answers
+    uint32_t ok;   // the thread is suspended until the phase completes or the time hint (in ns) has passed: no busy polling
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(kSuspendHintNs)
         : "memory");
     return ok != 0;
 }
 
-// Slow path of a bounded wait: polls until the phase completes, another role of this CTA has
-// given up, or about a second has passed; then it records which wait gave up (first writer
-// wins) and raises the CTA-wide flag.
+// Slow path of a bounded wait: sleeps on the barrier until the phase completes, another role of
+// this CTA has given up, or about a second has passed; then it records which wait gave up
+// (first writer wins) and raises the CTA-wide flag.
 __device__ __forceinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, Ctrl* c, uint32_t* status, uint32_t code) {
     long long t0 = 0;
-    uint32_t polls = 0;
 #pragma unroll 1
     while (!mbar_try(bar, parity)) {
-        __nanosleep(64);
-        if ((++polls & 63u) == 0u) {
-            if (c->abort_flag) return false;
-            const long long now = clock64();
-            if (t0 == 0) t0 = now;
-            if (now - t0 > kTimeoutCycles) {
-                atomicCAS(status, 0u, code | ((uint32_t)blockIdx.x << 8));
-                c->abort_flag = 1;
-                return false;
-            }
+        if (c->abort_flag) return false;
+        const long long now = clock64();
+        if (t0 == 0) t0 = now;
+        if (now - t0 > kTimeoutCycles) {
+            atomicCAS(status, 0u, code | ((uint32_t)blockIdx.x << 8));
+            c->abort_flag = 1;
+            return false;
         }
     }
     return true;
@@ -751,13 +748,15 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
         // columns into v.  consume<U>: wait for them, hand the slot back at once, fold them in; it also
         // asks whether the next slot is full already, an answer that is only needed after the FMAs.
         // With four promotion warps per scheduler the load of one warp hides behind the FMAs of the others.
-        const uint32_t tfull_s = smem_u32(&c->tfull[0]), tempty_s = smem_u32(&c->tempty[0]);
+        uint32_t tfull_s = smem_u32(&c->tfull[0]), tempty_s = smem_u32(&c->tempty[0]), tmem_row_r = tmem_row;
+        // opaque to the compiler: kept in registers instead of being recomputed from the thread index at every use
+        asm volatile("" : "+r"(tfull_s), "+r"(tempty_s), "+r"(tmem_row_r));
         auto request = [&](auto u_tag, bool ready) {
             constexpr uint32_t U = decltype(u_tag)::value;
             if (!__all_sync(0xffffffffu, ready)) ok = mbar_wait_warp(&c->tfull[U], p_full[U], c, a.status, 2u);
             p_full[U] ^= 1u;
             tc_fence_after();
-            tmem_ld32(tmem_row + U * kBN, v);
+            tmem_ld32(tmem_row_r + U * kBN, v);
         };
         auto consume = [&](auto u_tag, uint32_t scale_q, int k) -> bool {
             constexpr uint32_t U = decltype(u_tag)::value, N = (U + 1) & (kSlots - 1);
