@@ -141,7 +141,16 @@ def run_reference(args):
     if rank != 0:
         return
     case = workload(args.workload)
+    # a step is a bounded sample: at most 2048 rows, fewer when many steps are asked for, so that the
+    # whole run stays within about two minutes
     rows = 2048
+    t0 = time.perf_counter()
+    cpu_oracle_leg(case, rows)
+    t_leg = time.perf_counter() - t0
+    budget_s = 120.0
+    if (args.steps + args.warmup) * t_leg > budget_s:
+        rows = int(rows * budget_s / ((args.steps + args.warmup) * t_leg)) // 64 * 64
+        rows = max(64, rows)
     for _ in range(args.warmup):
         cpu_oracle_leg(case, rows)
     t0 = time.perf_counter()
@@ -176,6 +185,15 @@ def max_over_ranks(values, device, world):
 def whole_job_rate(units_per_rank, world, ms):
     """Units all ranks processed per second, given the slowest rank's time in milliseconds."""
     return world * units_per_rank / (ms * 1e-3)
+
+
+def graph_steps(K, nsets, cap=64):
+    """Steps per graph: the largest divisor of K that is a multiple of the buffer rotation and at
+    most `cap`; K itself (one graph, one replay) when there is none."""
+    for d in range(min(K, cap), 0, -1):
+        if K % d == 0 and d % nsets == 0:
+            return d
+    return K
 
 
 def run_tdq(args):
@@ -232,25 +250,52 @@ def run_tdq(args):
     if st != tdq.OK:
         raise RuntimeError("linear kernel reported a device-side timeout: 0x%x" % detail)
 
+    # The timed steps are replayed from a CUDA graph, so that the kernels run back to back and the
+    # device-side events between them measure kernels, not the host's launch path.  A graph holds
+    # G steps (a multiple of the buffer rotation, each with its own three events) and is replayed
+    # K / G times; per-kernel times come from the events of the last replay, the step time from
+    # the events around all replays.
+    G = graph_steps(args.steps, nsets) if not args.eager else 0
     sampler = ClockSampler(local)
+    launches0 = tdq.kernel_launch_count()
+    if G:
+        evs = [[torch.cuda.Event(enable_timing=True, external=True) for _ in range(3)] for _ in range(G)]
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for i in range(G):
+                step(args.warmup + i, evs[i])
+        launches_per_replay = tdq.kernel_launch_count() - launches0
+        graph.replay()                       # untimed: uploads the graph
+        barrier()
+        st, detail = tdq.workspace_status(wsp)
+        if st != tdq.OK:
+            raise RuntimeError("linear kernel reported a device-side timeout: 0x%x" % detail)
+    else:
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
-    launches0 = tdq.kernel_launch_count()
     barrier()
     t_begin = torch.cuda.Event(enable_timing=True)
     t_end = torch.cuda.Event(enable_timing=True)
     t_begin.record()
-    for i in range(args.steps):
-        step(args.warmup + i, evs[i])
+    if G:
+        for _ in range(args.steps // G):
+            graph.replay()
+    else:
+        for i in range(args.steps):
+            step(args.warmup + i, evs[i])
     t_end.record()
     barrier()
-    launches = tdq.kernel_launch_count() - launches0
+    if G:
+        launches = launches_per_replay * (args.steps // G)
+    else:
+        launches = tdq.kernel_launch_count() - launches0
     clocks = sampler.stop() if rank == 0 else None
     total_ms = t_begin.elapsed_time(t_end)
-    q_ms = sum(e[0].elapsed_time(e[1]) for e in evs)
-    l_ms = sum(e[1].elapsed_time(e[2]) for e in evs)
+    n_ev = len(evs)
+    q_ms = sum(e[0].elapsed_time(e[1]) for e in evs) * args.steps / n_ev
+    l_ms = sum(e[1].elapsed_time(e[2]) for e in evs) * args.steps / n_ev
 
     # end to end: pinned host X in, host Y out, through the host-buffer entry point
     xh = x_host.pin_memory()
@@ -315,6 +360,7 @@ def run_tdq(args):
                    config=dict(workload=case.name, x=[int(v) for v in case.x.shape], w=[int(v) for v in case.w.shape],
                                g=32, tau=1.0, zr=0.2, y_dtype="f32",
                                cache="rotating %d buffer sets, %.0f MB per step (L2 is 126 MB)" % (nsets, step_bytes / 1e6),
+                               launch=("CUDA graph of %d steps, replayed %d times" % (G, args.steps // G)) if G else "eager",
                                parallelism="rows sharded, %d replica(s)" % world),
                    kernels=dict(quantize_act=q_kernel, w4a4_linear=l_kernel,
                                 step_tokens_per_s=world * M * K / (total_ms * 1e-3)),
@@ -337,13 +383,16 @@ def run_tdq(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=None, help="default: 1000 (10 for --impl reference)")
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="tdq", choices=["tdq", "reference"])
     ap.add_argument("--workload", default="cfg4", choices=["cfg2", "cfg3", "cfg4"])
     ap.add_argument("--cpu-rows", type=int, default=18464)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--eager", action="store_true", help="launch every timed step from the host instead of replaying a CUDA graph")
     args = ap.parse_args()
+    if args.steps is None:
+        args.steps = 10 if args.impl == "reference" else 1000
     if args.impl == "reference":
         run_reference(args)
     else:
