@@ -455,7 +455,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
     const bool resident = a.a_resident != 0;
 
     if (t == 0) {
-        const uint32_t n_issuers = a.steps_per_grp == 1 ? 2u : 1u;   // MMA-issuing warps
+        const uint32_t n_issuers = a.steps_per_grp <= 2 ? 2u : 1u;   // MMA-issuing warps
         for (int i = 0; i < kMaxStages; ++i) { mbar_init(&c->full[i], 1); mbar_init(&c->empty[i], n_issuers); }
         for (int i = 0; i < kSlots; ++i) { mbar_init(&c->tfull[i], 1); mbar_init(&c->tempty[i], kPromoWarps); }
         mbar_init(&c->a_full, 1);
@@ -529,7 +529,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                     }
                 }
             }
-        } else if (warp == kMmaWarp || spg == 1) {
+        } else if (warp == kMmaWarp || spg <= 2) {
             // ------------------------------------------------------------ MMA issue (lane 0 issues)
             // A warp runs dependent scalar code at one instruction every few clocks, so this loop is
             // what paces the tensor pipe: everything that can be is hoisted, and the two cases are
@@ -545,8 +545,13 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
             const uint32_t tempty_s = smem_u32(&c->tempty[0]);
             const int n_steps = a.n_steps;
             // Group k of a tile uses TMEM slot k & 3, so a chunk of four steps always starts at slot 0.
-            auto role = [&](auto dual_tag) {
-                constexpr bool DUAL = decltype(dual_tag)::value;
+            // mode 0: one instruction per group, two warps that take the even and the odd slots (DUAL); 3: two
+            // instructions per group, two warps that take the first and the second group of a chunk (DUAL2);
+            // 1: groups of a multiple of four steps, so that a chunk belongs to one group and is issued as
+            // straight-line code (QUAD); 2: any other group width, one step at a time
+            auto role = [&](auto mode_tag) {
+                constexpr int MODE = decltype(mode_tag)::value;
+                constexpr bool DUAL = MODE == 0, QUAD = MODE == 1, DUAL2 = MODE == 3;
                 uint32_t s = 0, ph = 0, ic = 0;
                 bool ok = true;
                 // DUAL: this warp's two slots (me and me + 2), everything about them precomputed
@@ -593,6 +598,42 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                                 mma_issue_if<I8>(lane0 & act_b, tm_b, a_lo + off_b, b_lo + off_b, 0u);
                                 mma_commit_if(lane0 & act_b, tfull_b);
                                 q_b ^= act_b;
+                            } else if (DUAL2) {
+                                // group h of chunk c sits in slot 2 (c & 1) + h: this warp (h = me) alternates between its two slots
+                                const bool odd = (k0 & kChunk) != 0;
+                                const uint32_t act = 2 * me < (uint32_t)nk ? 1u : 0u;
+                                const uint32_t q = odd ? q_b : q_a;
+                                const bool rdy = mbar_test_s(odd ? tempty_b : tempty_a, q) || !act;
+                                if (!__all_sync(0xffffffffu, rdy)) {
+                                    ok = mbar_wait_warp(&c->tempty[me + (odd ? 2u : 0u)], q, c, a.status, 3u);
+                                    if (!ok) break;
+                                }
+                                tc_fence_after();
+                                const uint32_t d_tmem = odd ? tm_b : tm_a;
+                                mma_issue_if<I8>(lane0 & act, d_tmem, a_lo + 2 * off_a, b_lo + 2 * off_a, 0u);
+                                mma_issue_if<I8>(lane0 & act, d_tmem, a_lo + 2 * off_a + (kBlock >> 4), b_lo + 2 * off_a + (kBlock >> 4), 1u);
+                                mma_commit_if(lane0 & act, odd ? tfull_b : tfull_a);
+                                if (odd) q_b ^= act; else q_a ^= act;
+                            } else if (QUAD) {
+                                // all four steps of the chunk go to the same slot; n_steps is a multiple of four
+                                if (sub == 0 && !slot_ready) {
+                                    ok = mbar_wait_warp(&c->tempty[slot], (qm >> slot) & 1u, c, a.status, 3u);
+                                    if (!ok) break;
+                                }
+                                tc_fence_after();
+                                const uint32_t d_tmem = tmem_base + slot * kBN;
+                                mma_issue_if<I8>(lane0, d_tmem, a_lo, b_lo, sub == 0 ? 0u : 1u);
+                                mma_issue_if<I8>(lane0, d_tmem, a_lo + 1 * (kBlock >> 4), b_lo + 1 * (kBlock >> 4), 1u);
+                                mma_issue_if<I8>(lane0, d_tmem, a_lo + 2 * (kBlock >> 4), b_lo + 2 * (kBlock >> 4), 1u);
+                                mma_issue_if<I8>(lane0, d_tmem, a_lo + 3 * (kBlock >> 4), b_lo + 3 * (kBlock >> 4), 1u);
+                                sub += kChunk;
+                                if (sub == spg) {
+                                    sub = 0;
+                                    mma_commit_if(lane0, tfull_s + slot * 8);
+                                    qm ^= 1u << slot;
+                                    slot = (slot + 1) & (kSlots - 1);
+                                    slot_ready = __all_sync(0xffffffffu, mbar_test_s(tempty_s + slot * 8, (qm >> slot) & 1u));
+                                }
                             } else {
                                 uint32_t a_j = a_lo, b_j = b_lo;
 #pragma unroll 1
@@ -621,8 +662,10 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                     if (ok) mma_commit_if(lane0, smem_u32(&c->a_empty));
                 }
             };
-            if (spg == 1) role(std::true_type{});
-            else role(std::false_type{});
+            if (spg == 1) role(std::integral_constant<int, 0>{});
+            else if (spg == 2) role(std::integral_constant<int, 3>{});
+            else if (spg % kChunk == 0) role(std::integral_constant<int, 1>{});
+            else role(std::integral_constant<int, 2>{});
         }
     } else {
         setmaxnreg_inc<kRegsPromo>();
