@@ -719,40 +719,54 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
             w0 = ca < a.O ? __ldg(a.wscale + ca) : 0.f;
             b0 = (a.bias && ca < a.O) ? __ldg(a.bias + ca) : 0.f;
         };
+        bool store_pending = false;      // a staged tile whose bulk tensor store has not been started
+        int32_t store_x = 0, store_y = 0;
+        const int store_turn = (pw >> 2) * 4;   // group of the next tile at which this warp starts its store
+        auto issue_store = [&]() {
+            if (lane == 0) {
+                tma_store_2d(&ymap, strip_w, store_x, store_y);
+                bulk_commit_group();
+            }
+            store_pending = false;
+        };
         // y = (s_o * 2^e) * sum + bias for the tile that just finished, then on to the next tile
         auto finish_tile = [&]() {
+            if (store_pending) issue_store();            // a short tile: the previous store is still waiting for its turn
             if (lane == 0) bulk_wait_group_read0();      // the previous tile's store has read the strip
-            sts32(wsb_s + lane * 4, __float_as_uint(__fmul_rn(w0, a.out_scale)));
-            sts32(wsb_s + 128 + lane * 4, __float_as_uint(b0));
+            float* wsb = reinterpret_cast<float*>(smem_raw + (wsb_s - sm_s));
+            wsb[lane] = __fmul_rn(w0, a.out_scale);
+            wsb[32 + lane] = b0;
             __syncwarp();
+            uint8_t* strip = smem_raw + (strip_row - sm_s);
 #pragma unroll
             for (int j = 0; j < kCols / 4; ++j) {
                 float o0, o1, o2, o3;
                 unpack2(yacc[2 * j], o0, o1);
                 unpack2(yacc[2 * j + 1], o2, o3);
-                const uint4 s4 = lds128(wsb_s + j * 16), b4 = lds128(wsb_s + 128 + j * 16);
-                o0 = __fmaf_rn(__uint_as_float(s4.x), o0, __uint_as_float(b4.x));
-                o1 = __fmaf_rn(__uint_as_float(s4.y), o1, __uint_as_float(b4.y));
-                o2 = __fmaf_rn(__uint_as_float(s4.z), o2, __uint_as_float(b4.z));
-                o3 = __fmaf_rn(__uint_as_float(s4.w), o3, __uint_as_float(b4.w));
+                const float4 s4 = reinterpret_cast<const float4*>(wsb)[j], b4 = reinterpret_cast<const float4*>(wsb + 32)[j];
+                o0 = __fmaf_rn(s4.x, o0, b4.x);
+                o1 = __fmaf_rn(s4.y, o1, b4.y);
+                o2 = __fmaf_rn(s4.z, o2, b4.z);
+                o3 = __fmaf_rn(s4.w, o3, b4.w);
                 if (YBF16) {       // columns 4 j .. 4 j + 3: half of chunk j / 2
                     __nv_bfloat162 lo = __floats2bfloat162_rn(o0, o1);
                     __nv_bfloat162 hi = __floats2bfloat162_rn(o2, o3);
-                    sts64(strip_row + ((((uint32_t)j >> 1) ^ swz) << 4) + ((uint32_t)j & 1u) * 8,
-                          *reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+                    *reinterpret_cast<uint2*>(strip + ((((uint32_t)j >> 1) ^ swz) << 4) + ((uint32_t)j & 1u) * 8) =
+                        make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
                 } else {
-                    sts128(strip_row + (((uint32_t)j ^ swz) << 4), __float_as_uint(o0), __float_as_uint(o1),
-                           __float_as_uint(o2), __float_as_uint(o3));
+                    *reinterpret_cast<float4*>(strip + (((uint32_t)j ^ swz) << 4)) = make_float4(o0, o1, o2, o3);
                 }
             }
             const int64_t m0 = (int64_t)mt * kBM + quarter * 32;   // first row of this warp's block
             if (a.tma_ok) {
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes before the engine's reads
                 __syncwarp();
-                if (lane == 0 && m0 < a.M && n0 < a.O) {
-                    tma_store_2d(&ymap, strip_w, (int32_t)n0, (int32_t)m0);
-                    bulk_commit_group();
-                }
+                // The store is started a few groups into the next tile, each block of columns at its own
+                // time: sixteen warps that hand 4 KB to the copy engine at the same moment queue up behind
+                // one another, and starting a store blocks the warp until the engine has taken it.
+                store_pending = m0 < a.M && n0 < a.O;
+                store_x = (int32_t)n0;
+                store_y = (int32_t)m0;
             } else {          // any alignment: a row at a time, lane = column
                 __syncwarp();
                 const int rows = (int)min((int64_t)32, a.M - m0);
@@ -840,6 +854,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                 int k = 0;
 #pragma unroll 1
                 for (; k + 4 < Kg && ok; k += 4, scale_q += 4 * kScaleBlock) {   // four groups, and more behind them
+                    if (store_pending && k >= store_turn) issue_store();
                     request(u1, consume(u0, scale_q, k));
                     request(u2, consume(u1, scale_q, k));
                     request(u3, consume(u2, scale_q, k));
@@ -868,6 +883,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
             }
         }
         tmem_ld_wait();            // nothing may still be landing when TMEM is released
+        if (store_pending) issue_store();
         if (lane == 0) bulk_wait_group0();   // nor may a store still be reading this CTA's shared memory
     }
 
