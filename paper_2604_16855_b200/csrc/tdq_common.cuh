@@ -23,6 +23,25 @@ constexpr float kRoundMagic = 12582912.0f;
 
 extern std::atomic<uint64_t> g_launch_count;
 
+// The linear layer with either source of its A operand.  fx == nullptr: activation codes and
+// scales from memory (tdq_w4a4_linear).  Otherwise the activations themselves, quantized by the
+// GEMM's own producer; xcodes and xscale are ignored.
+struct FusedSrc {
+    const void* x;
+    int64_t row_stride;   // elements
+    bool bf16;
+    float seven_tau;
+    uint32_t flags;
+};
+tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* xscale, const uint8_t* wcodes,
+                       const float* wscale, const float* bias, int64_t M, int64_t I_pad, int64_t O, int32_t group_size,
+                       void* y, tdq_dtype y_dtype, int64_t y_row_stride, int32_t* acc_debug, void* workspace,
+                       size_t workspace_bytes, void* cuda_stream);
+// Argument checks of the quantizer and its fast-path conditions (tdq_quantize_act.cu).
+tdq_status check_act_args(const void* x, tdq_dtype dt, int64_t B, int64_t N, int64_t C, int64_t stride,
+                          const tdq_act_params* p);
+bool act_fast_path_ok(const void* x, tdq_dtype dt, int64_t C, int64_t stride, const tdq_act_params* p);
+
 inline tdq_status cuda_status(cudaError_t e) { return e == cudaSuccess ? TDQ_OK : TDQ_ERR_CUDA; }
 
 // Rank ceil(frac * g), 1-indexed, inside [1, g] (Supp. S2.2).  frac is a float, so a

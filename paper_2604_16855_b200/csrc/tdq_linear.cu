@@ -52,6 +52,7 @@
 #include <mutex>
 #include <type_traits>
 
+#include "tdq_act_group.cuh"
 #include "tdq_common.cuh"
 
 namespace tdq {
@@ -106,6 +107,11 @@ struct LinArgs {
     uint32_t* status;
     int32_t tma_ok;            // y can be written with bulk tensor stores (16-byte aligned base and row pitch)
     float out_scale;           // 2^18 (E4M3 route) or 2^-8 (int8 route)
+    // fused producer only: the activations themselves and the quantizer's parameters
+    const void* x;
+    int64_t x_stride;          // elements between rows of x
+    float seven_tau;
+    uint32_t act_flags;
 };
 
 struct Ctrl {
@@ -443,7 +449,10 @@ __device__ __noinline__ void debug_store(const LinArgs& a, const uint32_t* v, in
                 I8 ? ((int32_t)v[q] >> 8) : __float2int_rn(__uint_as_float(v[q]) * 262144.0f);
 }
 
-template <bool I8, bool YBF16, bool DBG>
+// FUSED: 0 the A operand comes as blocks from the workspace; 1 / 2: the promotion warps quantize the
+// work item's 128 rows of bf16 / fp32 activations themselves and write operand bytes and scales
+// straight into shared memory (A must be resident), so codes and scales never reach global memory.
+template <bool I8, bool YBF16, bool DBG, int FUSED = 0>
 __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a, const __grid_constant__ CUtensorMap ymap) {
     extern __shared__ __align__(128) uint8_t smem_raw[];   // no static shared memory: the window starts aligned
     Ctrl* c = reinterpret_cast<Ctrl*>(smem_raw);
@@ -458,7 +467,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
         const uint32_t n_issuers = a.steps_per_grp <= 2 ? 2u : 1u;   // MMA-issuing warps
         for (int i = 0; i < kMaxStages; ++i) { mbar_init(&c->full[i], 1); mbar_init(&c->empty[i], n_issuers); }
         for (int i = 0; i < kSlots; ++i) { mbar_init(&c->tfull[i], 1); mbar_init(&c->tempty[i], kPromoWarps); }
-        mbar_init(&c->a_full, 1);
+        mbar_init(&c->a_full, FUSED ? kPromoWarps : 1);
         mbar_init(&c->a_empty, n_issuers + kPromoWarps);
         c->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -490,7 +499,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
             for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++ic) {
                 const int mt = item / a.n_parts, part = item % a.n_parts;
                 const uint8_t* a_src = a.a_blocks + (int64_t)mt * a.n_steps * kBlock;
-                if (warp == 0) {
+                if (warp == 0 && !FUSED) {
                     ok = mbar_wait_warp(&c->a_empty, (ic & 1) ^ 1, c, a.status, 1u);
                     if (!ok) break;
                     if (lane == 0) {
@@ -708,7 +717,49 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
             nt_end = part_begin(part + 1);
             m = (int64_t)mt * kBM + row;
             row_ok = m < a.M;
-            ok = mbar_wait_warp(&c->a_full, ic & 1, c, a.status, 7u);
+            if (FUSED) {
+                // The previous item's A and scales are free once every MMA that read them has completed and
+                // every promotion warp has left the item (a_empty counts both).  Then thread = (row, group
+                // mod 4) quantizes its groups: Algorithm S1 steps 2-7 in registers, codes expanded to operand
+                // bytes in the block's core-matrix order, the step to the scale block.
+                ok = mbar_wait_warp(&c->a_empty, (ic & 1) ^ 1, c, a.status, 1u);
+                if (ok) {
+                    constexpr bool XBF = FUSED == 1;
+                    constexpr int kWords = XBF ? 16 : 32;
+                    const int pt = pw * 32 + lane, r = pt & (kBM - 1);
+                    const int64_t mr = (int64_t)mt * kBM + r;
+                    const uint32_t off = (uint32_t)((r >> 3) * 256 + (r & 7) * 16);
+                    for (int k = pt >> 7; k < a.Kg; k += kPromoWarps * 32 / kBM) {
+                        uint32_t out[4] = {0u, 0u, 0u, 0u};
+                        float delta = 0.0f;
+                        if (mr < a.M) {
+                            uint32_t w[kWords];
+                            const uint4* src = reinterpret_cast<const uint4*>(
+                                reinterpret_cast<const uint8_t*>(a.x) + ((size_t)mr * a.x_stride + (size_t)k * 32) * (XBF ? 2 : 4));
+#pragma unroll
+                            for (int q = 0; q < kWords / 4; ++q) {
+                                const uint4 t4 = __ldg(src + q);
+                                w[4 * q] = t4.x; w[4 * q + 1] = t4.y; w[4 * q + 2] = t4.z; w[4 * q + 3] = t4.w;
+                            }
+                            quantize_group32<XBF, 7>(w, a.seven_tau, a.act_flags, out, delta);
+                        }
+                        uint4 c0, c1;
+                        expand8<I8>(out[0], c0.x, c0.y);
+                        expand8<I8>(out[1], c0.z, c0.w);
+                        expand8<I8>(out[2], c1.x, c1.y);
+                        expand8<I8>(out[3], c1.z, c1.w);
+                        const uint32_t dst = ares_s + (uint32_t)k * kBlock + off;
+                        sts128(dst, c0.x, c0.y, c0.z, c0.w);
+                        sts128(dst + 128, c1.x, c1.y, c1.z, c1.w);
+                        sts32(scales_s + (uint32_t)k * kScaleBlock + (uint32_t)r * 4, __float_as_uint(delta));
+                    }
+                    // written through the generic proxy, read by the tensor core through the async proxy
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    mbar_arrive_lane0(&c->a_full, lane);
+                }
+            }
+            if (ok) ok = mbar_wait_warp(&c->a_full, ic & 1, c, a.status, 7u);
         };
         auto begin_tile = [&]() {
             n0 = (int64_t)nt * kBN + col0;
@@ -1007,12 +1058,15 @@ extern "C" size_t tdq_linear_workspace_bytes(int64_t M, int64_t I_pad, int64_t O
     return kWorkspaceHeader + p.a_bytes + p.b_bytes + p.s_bytes;
 }
 
-extern "C" tdq_status tdq_w4a4_linear(const uint8_t* xcodes, const float* xscale, const uint8_t* wcodes,
-                                      const float* wscale, const float* bias, int64_t M, int64_t I_pad, int64_t O,
-                                      int32_t group_size, void* y, tdq_dtype y_dtype, int64_t y_row_stride,
-                                      int32_t* acc_debug, void* workspace, size_t workspace_bytes,
-                                      void* cuda_stream) {
-    if (!xcodes || !xscale || !wcodes || !wscale || !y) return TDQ_ERR_INVALID_ARG;
+namespace tdq {
+
+tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* xscale, const uint8_t* wcodes,
+                       const float* wscale, const float* bias, int64_t M, int64_t I_pad, int64_t O, int32_t group_size,
+                       void* y, tdq_dtype y_dtype, int64_t y_row_stride, int32_t* acc_debug, void* workspace,
+                       size_t workspace_bytes, void* cuda_stream) {
+    if (!fx && (!xcodes || !xscale)) return TDQ_ERR_INVALID_ARG;
+    if (fx && (!fx->x || group_size != 32 || acc_debug)) return TDQ_ERR_UNSUPPORTED;
+    if (!wcodes || !wscale || !y) return TDQ_ERR_INVALID_ARG;
     if (M < 0 || O <= 0 || I_pad <= 0 || y_row_stride < O) return TDQ_ERR_INVALID_ARG;
     if (y_dtype != TDQ_F32 && y_dtype != TDQ_BF16) return TDQ_ERR_INVALID_ARG;
     if (group_size <= 0 || I_pad % group_size) return TDQ_ERR_INVALID_ARG;
@@ -1021,7 +1075,7 @@ extern "C" tdq_status tdq_w4a4_linear(const uint8_t* xcodes, const float* xscale
     Plan p;
     if (!make_plan(M, I_pad, O, group_size, 148, p)) return TDQ_ERR_UNSUPPORTED;
     if (!workspace || workspace_bytes < kWorkspaceHeader + p.a_bytes + p.b_bytes + p.s_bytes) return TDQ_ERR_WORKSPACE;
-    if (reinterpret_cast<uintptr_t>(xcodes) % 16 || reinterpret_cast<uintptr_t>(wcodes) % 16 ||
+    if ((!fx && reinterpret_cast<uintptr_t>(xcodes) % 16) || reinterpret_cast<uintptr_t>(wcodes) % 16 ||
         reinterpret_cast<uintptr_t>(workspace) % 16)
         return TDQ_ERR_ALIGNMENT;
     if (M == 0) return TDQ_OK;
@@ -1029,6 +1083,7 @@ extern "C" tdq_status tdq_w4a4_linear(const uint8_t* xcodes, const float* xscale
     const int n_sm = sm_count();
     if (n_sm <= 0) return TDQ_ERR_CUDA;
     if (!make_plan(M, I_pad, O, group_size, n_sm, p)) return TDQ_ERR_UNSUPPORTED;
+    if (fx && !p.a_resident) return TDQ_ERR_UNSUPPORTED;   // the fused producer writes a whole row block's A into shared memory
 
     uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
     const bool i8 = group_size > 32;   // several instructions chain into one slot: keep the integer accumulator
@@ -1043,14 +1098,15 @@ extern "C" tdq_status tdq_w4a4_linear(const uint8_t* xcodes, const float* xscale
     e.n_steps = p.n_steps; e.n_chunks = p.n_chunks;
     e.steps_per_grp = group_size / 32;
     e.Kg = p.Kg;
-    e.tiles_m = (int32_t)p.tiles_m; e.tiles_n = (int32_t)p.tiles_n;
+    e.tiles_m = fx ? 0 : (int32_t)p.tiles_m;   // fused: only the weights are expanded
+    e.tiles_n = (int32_t)p.tiles_n;
 
     LinArgs a;
     a.a_blocks = e.a_blocks; a.b_blocks = e.b_blocks; a.s_blocks = e.s_blocks;
     a.wscale = wscale; a.bias = bias;
     a.M = M; a.O = O;
     a.n_steps = p.n_steps; a.steps_per_grp = e.steps_per_grp; a.Kg = p.Kg;
-    a.tiles_m = e.tiles_m; a.tiles_n = e.tiles_n; a.n_parts = p.n_parts;
+    a.tiles_m = (int32_t)p.tiles_m; a.tiles_n = e.tiles_n; a.n_parts = p.n_parts;
     a.a_resident = p.a_resident; a.n_stages = p.n_stages;
     a.ares_off = p.ares_off; a.ring_off = p.ring_off; a.stage_bytes = p.stage_bytes;
     a.staging_off = p.staging_off;
@@ -1065,6 +1121,10 @@ extern "C" tdq_status tdq_w4a4_linear(const uint8_t* xcodes, const float* xscale
         encode_y_map(&ymap, y, y_dtype == TDQ_BF16, M, O, y_row_stride))
         a.tma_ok = 1;
     a.out_scale = i8 ? 0.00390625f : 262144.0f;
+    a.x = fx ? fx->x : nullptr;
+    a.x_stride = fx ? fx->row_stride : 0;
+    a.seven_tau = fx ? fx->seven_tau : 0.0f;
+    a.act_flags = fx ? fx->flags : 0u;
 
     const bool ybf = y_dtype == TDQ_BF16, dbg = acc_debug != nullptr;
     void (*kernel)(LinArgs, CUtensorMap) = nullptr;
@@ -1072,11 +1132,15 @@ extern "C" tdq_status tdq_w4a4_linear(const uint8_t* xcodes, const float* xscale
     TDQ_PICK(false, false, false) TDQ_PICK(false, true, false) TDQ_PICK(true, false, false) TDQ_PICK(true, true, false)
     TDQ_PICK(false, false, true) TDQ_PICK(false, true, true) TDQ_PICK(true, false, true) TDQ_PICK(true, true, true)
 #undef TDQ_PICK
+    if (fx) {
+        if (fx->bf16) kernel = ybf ? w4a4_gemm_kernel<false, true, false, 1> : w4a4_gemm_kernel<false, false, false, 1>;
+        else kernel = ybf ? w4a4_gemm_kernel<false, true, false, 2> : w4a4_gemm_kernel<false, false, false, 2>;
+    }
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess)
         return TDQ_ERR_CUDA;
     if (cudaMemsetAsync(workspace, 0, 16, stream) != cudaSuccess) return TDQ_ERR_CUDA;
 
-    const unsigned pieces = (unsigned)((p.tiles_m + p.tiles_n) * p.n_chunks);
+    const unsigned pieces = (unsigned)((e.tiles_m + e.tiles_n) * p.n_chunks);
     if (i8)
         expand_kernel<true><<<pieces, kExpandThreads, 0, stream>>>(e);
     else
@@ -1090,6 +1154,17 @@ extern "C" tdq_status tdq_w4a4_linear(const uint8_t* xcodes, const float* xscale
     if (cudaGetLastError() != cudaSuccess) return TDQ_ERR_CUDA;
     g_launch_count.fetch_add(1, std::memory_order_relaxed);
     return TDQ_OK;
+}
+
+}  // namespace tdq
+
+extern "C" tdq_status tdq_w4a4_linear(const uint8_t* xcodes, const float* xscale, const uint8_t* wcodes,
+                                      const float* wscale, const float* bias, int64_t M, int64_t I_pad, int64_t O,
+                                      int32_t group_size, void* y, tdq_dtype y_dtype, int64_t y_row_stride,
+                                      int32_t* acc_debug, void* workspace, size_t workspace_bytes,
+                                      void* cuda_stream) {
+    return linear_impl(nullptr, xcodes, xscale, wcodes, wscale, bias, M, I_pad, O, group_size, y, y_dtype, y_row_stride,
+                       acc_debug, workspace, workspace_bytes, cuda_stream);
 }
 
 extern "C" tdq_status tdq_workspace_status(const void* workspace, void* cuda_stream, uint32_t* detail) {
@@ -1121,7 +1196,7 @@ extern "C" tdq_status tdq_w4a4_linear_static(const uint8_t* xcodes, const float*
                                              int64_t O, int32_t group_size, void* y, tdq_dtype y_dtype,
                                              int64_t y_row_stride, int32_t wait, void* cuda_stream) {
     // the argument checks that do not depend on the scratch come first, as in tdq_w4a4_linear
-    if (!xcodes || !xscale || !wcodes || !wscale || !y) return TDQ_ERR_INVALID_ARG;
+    if (!wcodes || !wscale || !y) return TDQ_ERR_INVALID_ARG;
     if (M < 0 || O <= 0 || I_pad <= 0 || y_row_stride < O) return TDQ_ERR_INVALID_ARG;
     if (group_size <= 0 || I_pad % group_size) return TDQ_ERR_INVALID_ARG;
     if (group_size % 32 || group_size > 4096) return TDQ_ERR_UNSUPPORTED;

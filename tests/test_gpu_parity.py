@@ -221,3 +221,63 @@ def test_sweep_layers_spot_check(tdq):
         x = case.x.reshape(-1, case.C)[:512]
         y, ref = _linear_case(tdq, x, True, case.w, want_acc=False)
         compare_y(y, ref, case.C // 32)
+
+
+# ------------------------------------------------------------------------------------------
+# fused variant: the quantizer as the producer of the linear layer's A operand
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("idx,rows,bf16_x,out_dtype,use_bias", [
+    (1, None, False, torch.float32, False),     # cfg1: fp32 activations, two groups per row
+    (2, 3000, True, torch.float32, True),       # cfg2: several row blocks per CTA, ragged last block
+    (3, 1500, True, torch.float32, False),      # cfg3: ten groups per row (a ragged last quad)
+    (3, 700, True, torch.bfloat16, True),
+    (4, 400, True, torch.float32, False),       # cfg4: the widest contraction that stays resident
+])
+def test_fused_matches_oracle_and_the_two_call_path(tdq, idx, rows, bf16_x, out_dtype, use_bias):
+    case = getattr(si, "config%d" % idx)()
+    x = case.x.reshape(-1, case.C)
+    if rows:
+        x = x[:rows]
+    xt = to_cuda(x, bf16=bf16_x)
+    wc, ws = tdq.quantize_weight(to_cuda(case.w))
+    bias_np = (np.linspace(-1.0, 1.0, case.O).astype(np.float32) * 0.01) if use_bias else None
+    bias = torch.from_numpy(bias_np).cuda() if use_bias else None
+    y = tdq.quant_linear_fused(xt, wc, ws, bias, out_dtype=out_dtype)
+    codes, scale = tdq.quantize_act(xt)
+    y2 = tdq.w4a4_linear(codes, scale, wc, ws, bias, out_dtype=out_dtype)
+    # the same kernel consumes the same operand bytes and scales: bit-identical results
+    assert torch.equal(y.view(torch.int16 if out_dtype == torch.bfloat16 else torch.int32),
+                       y2.view(torch.int16 if out_dtype == torch.bfloat16 else torch.int32))
+    if out_dtype == torch.float32:
+        xa = oracle.quantize_act(_f32(x, bf16_x))
+        wq = oracle.quantize_weight(case.w)
+        ref = oracle.w4a4_linear(xa["codes"], xa["scale"], wq["codes"], wq["scale"], bias=bias_np)
+        compare_y(y.cpu().numpy(), ref, case.C // 32)
+
+
+@pytest.mark.gpu
+def test_fused_settings_and_refusals(tdq):
+    case = si.config3()
+    x = case.x.reshape(-1, case.C)[:300]
+    xt = to_cuda(x, bf16=True)
+    wc, ws = tdq.quantize_weight(to_cuda(case.w))
+    # C1 binding (small tau), C2 off, both off: the producer follows the same flags as the quantizer
+    for tau, flags in [(0.25, 3), (1.0, 1), (1.0, 0)]:
+        p = tdq.act_params(tau=tau, flags=flags)
+        y = tdq.quant_linear_fused(xt, wc, ws, params=p)
+        codes, scale = tdq.quantize_act(xt, p)
+        y2 = tdq.w4a4_linear(codes, scale, wc, ws)
+        assert torch.equal(y.view(torch.int32), y2.view(torch.int32))
+    # refused: another zero-bin rank, another group size, a contraction too wide to stay in shared memory
+    with pytest.raises(tdq.TdqError) as e:
+        tdq.quant_linear_fused(xt, wc, ws, params=tdq.act_params(zr=0.5))
+    assert e.value.code == tdq.ERR_UNSUPPORTED
+    with pytest.raises(tdq.TdqError) as e:
+        tdq.quant_linear_fused(xt, wc, ws, params=tdq.act_params(g=64))
+    assert e.value.code == tdq.ERR_UNSUPPORTED
+    wide = torch.zeros((64, 2048), dtype=torch.bfloat16, device="cuda")
+    wcw, wsw = tdq.quantize_weight(torch.zeros((32, 2048), device="cuda"))
+    with pytest.raises(tdq.TdqError) as e:
+        tdq.quant_linear_fused(wide, wcw, wsw)
+    assert e.value.code == tdq.ERR_UNSUPPORTED
