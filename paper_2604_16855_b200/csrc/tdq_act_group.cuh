@@ -251,5 +251,78 @@ __device__ __forceinline__ void quantize_group32(const uint32_t (&w)[BF16 ? 16 :
 }
 
 
+// The same result as quantize_group32<., 7> with a small register footprint, for callers that have
+// few registers to spare: the group (64 or 128 bytes at src, 16-byte aligned) is read twice instead
+// of being held in registers, and the seven smallest magnitudes are kept by insertion.  Every
+// quantity that reaches the output is computed by the same operations in the same precision; only
+// the screen that decides whether the exact deviation is needed differs, and both screens are safe.
+template <bool BF16>
+__device__ __forceinline__ void quantize_group32_lean(const uint4* src, float seven_tau, uint32_t flags,
+                                                      uint32_t (&out)[4], float& delta) {
+    constexpr int kChunks = BF16 ? 4 : 8;           // 16-byte chunks of the group
+    constexpr int kPer = 32 / kChunks;              // elements per chunk
+    auto elem = [](const uint4& t, int e) -> float {
+        const uint32_t w[4] = {t.x, t.y, t.z, t.w};
+        if (BF16) return (e & 1) ? __uint_as_float(w[e >> 1] & 0xffff0000u) : __uint_as_float(w[e >> 1] << 16);
+        return __uint_as_float(w[e]);
+    };
+    uint32_t small[7];                              // the seven smallest |x| so far (binary32 bit patterns), ascending
+#pragma unroll
+    for (int j = 0; j < 7; ++j) small[j] = 0x7f800000u;
+    uint32_t kmax = 0u;
+    float s1 = 0.0f, s2 = 0.0f;
+#pragma unroll 1
+    for (int q = 0; q < kChunks; ++q) {
+        const uint4 t = __ldg(src + q);
+#pragma unroll
+        for (int e = 0; e < kPer; ++e) {
+            const float x = elem(t, e);
+            uint32_t key = __float_as_uint(x) & 0x7fffffffu;
+            kmax = max(kmax, key);
+            s1 += x;
+            s2 = fmaf(x, x, s2);
+#pragma unroll
+            for (int j = 0; j < 7; ++j) {
+                const uint32_t lo = min(small[j], key);
+                key = max(small[j], key);
+                small[j] = lo;
+            }
+        }
+    }
+    const float c_base = __uint_as_float(kmax);
+    const float thr = (flags & TDQ_ENABLE_C2) ? __uint_as_float(small[6]) : 0.0f;
+    float sigma = INFINITY;                         // an idle C1 bound
+    if (flags & TDQ_ENABLE_C1) {
+        float cmin = c_base;
+        if (flags & TDQ_ENABLE_C2) cmin = fminf(cmin, __fmul_rn(14.0f, thr));
+        if (!c1_cannot_bind(s1, s2, seven_tau, cmin)) {
+            auto get = [&](int i) -> float {
+                if (BF16) return __uint_as_float((uint32_t)__ldg(reinterpret_cast<const uint16_t*>(src) + i) << 16);
+                return __ldg(reinterpret_cast<const float*>(src) + i);
+            };
+            sigma = sigma_exact32(get);
+        }
+    }
+    float c;
+    dcrp_project(c_base, sigma, thr, seven_tau, flags, c, delta);
+    const bool fast = delta <= 1e30f;               // otherwise 1 / Delta would be subnormal: take the IEEE division
+    const float rcp = fast ? __frcp_rn(delta) : 0.0f;
+#pragma unroll
+    for (int wd = 0; wd < 4; ++wd) {
+        uint32_t acc = 0u;
+#pragma unroll
+        for (int h = 0; h < 8 / kPer; ++h) {
+            const uint4 t = __ldg(src + wd * (8 / kPer) + h);
+#pragma unroll
+            for (int e = 0; e < kPer; ++e) {
+                const float x = elem(t, e);
+                const uint32_t nib = fast ? nibble_fast(x, c, delta, rcp) : nibble_ieee(x, c, delta);
+                acc |= nib << (4 * (h * kPer + e));
+            }
+        }
+        out[wd] = acc;
+    }
+}
+
 }  // namespace
 }  // namespace tdq

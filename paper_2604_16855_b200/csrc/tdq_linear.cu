@@ -725,24 +725,17 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                 ok = mbar_wait_warp(&c->a_empty, (ic & 1) ^ 1, c, a.status, 1u);
                 if (ok) {
                     constexpr bool XBF = FUSED == 1;
-                    constexpr int kWords = XBF ? 16 : 32;
                     const int pt = pw * 32 + lane, r = pt & (kBM - 1);
                     const int64_t mr = (int64_t)mt * kBM + r;
                     const uint32_t off = (uint32_t)((r >> 3) * 256 + (r & 7) * 16);
                     for (int k = pt >> 7; k < a.Kg; k += kPromoWarps * 32 / kBM) {
                         uint32_t out[4] = {0u, 0u, 0u, 0u};
                         float delta = 0.0f;
-                        if (mr < a.M) {
-                            uint32_t w[kWords];
-                            const uint4* src = reinterpret_cast<const uint4*>(
-                                reinterpret_cast<const uint8_t*>(a.x) + ((size_t)mr * a.x_stride + (size_t)k * 32) * (XBF ? 2 : 4));
-#pragma unroll
-                            for (int q = 0; q < kWords / 4; ++q) {
-                                const uint4 t4 = __ldg(src + q);
-                                w[4 * q] = t4.x; w[4 * q + 1] = t4.y; w[4 * q + 2] = t4.z; w[4 * q + 3] = t4.w;
-                            }
-                            quantize_group32<XBF, 7>(w, a.seven_tau, a.act_flags, out, delta);
-                        }
+                        if (mr < a.M)
+                            quantize_group32_lean<XBF>(
+                                reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(a.x) +
+                                                               ((size_t)mr * a.x_stride + (size_t)k * 32) * (XBF ? 2 : 4)),
+                                a.seven_tau, a.act_flags, out, delta);
                         uint4 c0, c1;
                         expand8<I8>(out[0], c0.x, c0.y);
                         expand8<I8>(out[1], c0.z, c0.w);
