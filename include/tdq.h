@@ -116,10 +116,18 @@ tdq_status tdq_w4a4_linear(const uint8_t* xcodes, const float* xscale, const uin
                            void* cuda_stream);
 
 /*
- * Quantizer fused into the linear layer as the producer of its A operand: same result as
- * tdq_quantize_act followed by tdq_w4a4_linear, but activation codes and scales never
- * reach global memory.  Requires group_size == 32, C % 32 == 0 and the fast-path
- * alignment of tdq_quantize_act; otherwise TDQ_ERR_UNSUPPORTED.
+ * Quantizer fused into the linear layer as the producer of its A operand (the paper's remark
+ * that the method needs "no additional activation pass", Sec. 4, taken literally): the same
+ * result, bit for bit, as tdq_quantize_act followed by tdq_w4a4_linear, but activation codes
+ * and scales never reach global memory.  For every block of 128 token rows the kernel
+ * quantizes the rows into shared memory and keeps them there for all output columns.
+ *   x, B, N, C, row_stride_elems, p   as for tdq_quantize_act;   wcodes [O, C/2], wscale [O],
+ *   bias NULL or [O];   y, y_dtype, y_row_stride, workspace as for tdq_w4a4_linear
+ *   (workspace size: tdq_linear_workspace_bytes(B*N, C, O, 32)).
+ * TDQ_ERR_UNSUPPORTED unless: group_size == 32, C % 32 == 0, base_percentile == 1, x 16-byte
+ * aligned with a row pitch that is a multiple of 16 bytes, the zero-bin rank ceil(32 zr) == 7
+ * when the C2 bound is enabled, and C <= 768 (a row block's operand bytes must fit in shared
+ * memory).  Callers fall back to the two calls in those cases.
  */
 tdq_status tdq_quant_linear_fused(const void* x, tdq_dtype x_dtype, int64_t B, int64_t N, int64_t C,
                                   int64_t row_stride_elems, const tdq_act_params* p /* HOST */,
