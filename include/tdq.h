@@ -116,8 +116,8 @@ tdq_status tdq_w4a4_linear(const uint8_t* xcodes, const float* xscale, const uin
                            void* cuda_stream);
 
 /*
- * Quantizer fused into the linear layer as the producer of its A operand (the paper's remark
- * that the method needs "no additional activation pass", Sec. 4, taken literally): the same
+ * Quantizer fused into the linear layer as the producer of its A operand (Algorithm S1 steps
+ * 1-10 in one kernel, with no pass over the activations besides the layer's own): the same
  * result, bit for bit, as tdq_quantize_act followed by tdq_w4a4_linear, but activation codes
  * and scales never reach global memory.  For every block of 128 token rows the kernel
  * quantizes the rows into shared memory and keeps them there for all output columns.
