@@ -196,6 +196,97 @@ def graph_steps(K, nsets, cap=64):
     return K
 
 
+def time_graph(fn, n_inner, replays=5):
+    """Captures n_inner calls of fn(i) into a CUDA graph, replays it, returns ms per call (device events)."""
+    import torch
+    fn(0)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for i in range(n_inner):
+            fn(i)
+    g.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(replays):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / (replays * n_inner)
+
+
+def fused_leg(tdq, xs, wcodes, wscale, ys, wsp, M, C, O, esize):
+    """The fused entry point on the same workload and buffer rotation: ms per call and its bytes."""
+    n = len(xs)
+    ms = time_graph(lambda i: tdq.quant_linear_fused(xs[i % n], wcodes, wscale, y=ys[i % n], workspace=wsp), 4 * n)
+    bytes_ = M * C * esize + O * C // 2 + O * 4 + M * O * 4
+    return dict(name="tdq_quant_linear_fused", ms=ms, gbs=bytes_ / (ms * 1e-3) / 1e9, tops=2.0 * M * C * O / (ms * 1e-3) / 1e12,
+                algorithmic_bytes=bytes_)
+
+
+def sweep_leg(tdq, dev):
+    """The 32-layer sweep (two blocks of qkv, proj, fc1, fc2 in each of four encoder stages, batch 8): every layer
+    quantizes its own input and runs its linear layer; total time per pass, launched from the host and from a graph."""
+    import torch
+    import synth_inputs as si
+    layers = []
+    max_y = max_codes = max_scale = max_ws = 0
+    for li in range(32):
+        case = si.config5_layer(li, batch=8)
+        x = torch.from_numpy(case.x.reshape(case.M, case.C).view(np.int16).copy()).view(torch.bfloat16).to(dev)
+        wc, ws = tdq.quantize_weight(torch.from_numpy(case.w).to(dev), 32)
+        layers.append((x, wc, ws, case.M, case.C, case.O))
+        max_y = max(max_y, case.M * case.O)
+        max_codes = max(max_codes, case.M * case.C // 2)
+        max_scale = max(max_scale, case.M * case.C // 32)
+        max_ws = max(max_ws, tdq.linear_workspace(case.M, case.C, case.O, 32, dev).numel())
+    ybuf = torch.empty((max_y,), dtype=torch.float32, device=dev)
+    cbuf = torch.empty((max_codes,), dtype=torch.uint8, device=dev)
+    sbuf = torch.empty((max_scale,), dtype=torch.float32, device=dev)
+    wsp = torch.empty((max_ws,), dtype=torch.uint8, device=dev)
+    params = tdq.default_act_params()
+
+    def one_pass(_=0):
+        for (x, wc, ws, M, C, O) in layers:
+            codes = cbuf[:M * C // 2].view(M, C // 2)
+            scale = sbuf[:M * C // 32].view(M, C // 32)
+            tdq.quantize_act(x, params, codes=codes, scale=scale)
+            tdq.w4a4_linear(codes, scale, wc, ws, y=ybuf[:M * O].view(M, O), workspace=wsp)
+
+    def one_pass_fused(_=0):
+        n_two = 0
+        for (x, wc, ws, M, C, O) in layers:
+            if C <= 768:
+                tdq.quant_linear_fused(x, wc, ws, y=ybuf[:M * O].view(M, O), workspace=wsp)
+            else:                     # the fused kernel keeps a row block's operand in shared memory: C <= 768
+                codes = cbuf[:M * C // 2].view(M, C // 2)
+                scale = sbuf[:M * C // 32].view(M, C // 32)
+                tdq.quantize_act(x, params, codes=codes, scale=scale)
+                tdq.w4a4_linear(codes, scale, wc, ws, y=ybuf[:M * O].view(M, O), workspace=wsp)
+                n_two += 1
+        return n_two
+
+    for _ in range(3):
+        one_pass()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(5):
+        one_pass()
+    e1.record()
+    torch.cuda.synchronize()
+    eager_ms = e0.elapsed_time(e1) / 5
+    graph_ms = time_graph(one_pass, 1)
+    n_two = one_pass_fused()
+    fused_ms = time_graph(one_pass_fused, 1)
+    macs = sum(M * C * O for (_, _, _, M, C, O) in layers)
+    xbytes = sum(M * C * 2 for (_, _, _, M, C, O) in layers)
+    ybytes = sum(M * O * 4 for (_, _, _, M, C, O) in layers)
+    return dict(layers=32, batch=8, eager_us=eager_ms * 1e3, graph_us=graph_ms * 1e3, fused_graph_us=fused_ms * 1e3,
+                fused_layers=32 - n_two, macs=macs, x_bytes=xbytes, y_bytes=ybytes,
+                graph_tops=2.0 * macs / (graph_ms * 1e-3) / 1e12, graph_gbs=(xbytes + ybytes) / (graph_ms * 1e-3) / 1e9)
+
+
 def run_tdq(args):
     import torch
     import torch.distributed as dist
@@ -325,6 +416,12 @@ def run_tdq(args):
     e2e_ms = e0.elapsed_time(e1)
 
     total_ms, q_ms, l_ms, e2e_ms = max_over_ranks([total_ms, q_ms, l_ms, e2e_ms], dev, world)
+    fused = sweep = None
+    if world == 1 and not args.no_extras:
+        fused = fused_leg(tdq, xs, wcodes, wscale, ys, wsp, M, C, O, esize)
+        del xs, codes, scales, ys
+        torch.cuda.empty_cache()
+        sweep = sweep_leg(tdq, dev)
 
     if rank == 0:
         peaks = load_peaks()
@@ -362,7 +459,7 @@ def run_tdq(args):
                                cache="rotating %d buffer sets, %.0f MB per step (L2 is 126 MB)" % (nsets, step_bytes / 1e6),
                                launch=("CUDA graph of %d steps, replayed %d times" % (G, args.steps // G)) if G else "eager",
                                parallelism="rows sharded, %d replica(s)" % world),
-                   kernels=dict(quantize_act=q_kernel, w4a4_linear=l_kernel,
+                   kernels=dict(quantize_act=q_kernel, w4a4_linear=l_kernel, fused=fused, sweep_cfg5=sweep,
                                 step_tokens_per_s=world * M * K / (total_ms * 1e-3)),
                    roofline=roof, clocks=clocks, gpu_launches=int(launches),
                    e2e=dict(value=e2e_value, unit="GB/s", ms_per_step=e2e_ms / e2e_steps,
@@ -389,6 +486,7 @@ def main():
     ap.add_argument("--workload", default="cfg4", choices=["cfg2", "cfg3", "cfg4"])
     ap.add_argument("--cpu-rows", type=int, default=18464)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the fused-call and 32-layer sweep legs")
     ap.add_argument("--eager", action="store_true", help="launch every timed step from the host instead of replaying a CUDA graph")
     args = ap.parse_args()
     if args.steps is None:
