@@ -41,6 +41,11 @@ METRIC = "quantizer GB/s and W4A4 linear TOPS at 1 B200, % of HBM / INT8 rooflin
 L2_BYTES = 126 * 2 ** 20
 
 
+# DRAM bytes (read + write) of one w4a4_gemm_kernel launch on cfg4 from the ncu capture summarised in
+# profiles/w4a4_gemm_kernel_cfg4.md; reported only for that workload and output type.
+GEMM_DRAM_TRAFFIC_CFG4 = 185.5e6
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -441,7 +446,8 @@ def run_tdq(args):
         if l_ms >= q_ms:
             if l_kernel["bound"] == "hbm":
                 roof = dict(kernel="tdq_w4a4_linear", bound="hbm", achieved=l_gbs, peak=peaks["hbm_gbs"],
-                            unit="GB/s", frac=l_gbs / peaks["hbm_gbs"], traffic=None)
+                            unit="GB/s", frac=l_gbs / peaks["hbm_gbs"],
+                            traffic=GEMM_DRAM_TRAFFIC_CFG4 if case.name.startswith("cfg4") else None)
             else:
                 roof = dict(kernel="tdq_w4a4_linear", bound="tensor", achieved=l_tops, peak=int8_peak,
                             unit="TOP/s", frac=l_tops / int8_peak, traffic=None)
