@@ -31,19 +31,29 @@
 //      moves operands with plain 1-D bulk copies (cp.async.bulk + mbarrier) and no tensor maps.
 //   2. w4a4_gemm_kernel   persistent, one CTA per SM, 128 x 128 output tiles.  Warp roles:
 //        warps 0-1   producers: one lane each issues the bulk copies of alternate ring stages
-//        warp  2     one lane issues the MMAs and the commits that release buffers
+//        warps 2-3   MMA issue and the commits that release buffers.  Group k of a tile uses TMEM slot
+//                    k & 3.  The issue loop is straight-line, predicated code (a lone warp runs
+//                    dependent scalar code slowly, and branches cost most): at g = 32 the two warps take
+//                    the even and the odd slots, at g = 64 the first and the second group of a stage,
+//                    at g a multiple of 128 warp 2 issues a stage's four steps in a row.
 //        warps 4-19  promotion + epilogue: warp w owns TMEM lanes 32 (w % 4).. (its rows) and 32
 //                    columns; a thread keeps 32 float accumulators of one output row and one
 //                    32-value landing buffer.  Sixteen warps, four per scheduler: a warp executes
 //                    dependent instructions only every few clocks, so the TMEM load and the
-//                    barrier traffic of one warp hide behind the FMAs of the other three.
+//                    barrier traffic of one warp hide behind the FMAs of the other three.  The loop
+//                    is unrolled over the four slots, so slot, barrier and TMEM addresses are constants.
 //      A work item is one 128-row block of A with a range of column tiles.  The item's scales,
 //      and its A block when the whole K extent fits, are loaded once per item; B (and A
 //      otherwise) streams through a ring of stages of 4 K-steps.  TMEM holds four 128-column
 //      accumulator slots, each with a full/empty mbarrier pair.
-//      In the epilogue every thread parks its 32 outputs in its own shared-memory strip; the
-//      promotion warps then read the tile back row by row, so that one warp instruction stores
-//      512 contiguous bytes of y.
+//      In the epilogue a warp needs no other warp: every thread scales its 32 sums and parks them in
+//      the warp's own 4 KB strip of shared memory, laid out (and swizzled) as the source box of a
+//      bulk tensor store; lane 0 starts one 32 x 32 store per tile, a few groups into the next
+//      tile, and the copy engine clips it at the edges of y.  Unaligned y is written element by
+//      element from the same strip.
+//   The fused instantiation (tdq_quant_linear_fused) replaces the load of an item's A block and
+//   scales: the promotion warps quantize the item's 128 activation rows into the same shared-memory
+//   regions before they start on its tiles.
 //
 // Every wait on an mbarrier is bounded: after about a second the thread records a code in the
 // workspace status word and raises a CTA-wide flag; every role then leaves its loops, the CTA
@@ -176,13 +186,6 @@ __device__ __forceinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, C
     return true;
 }
 
-// Bounded wait by one thread: false when the phase did not complete in time.  `code` names the
-// wait in the status word.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Ctrl* c, uint32_t* status, uint32_t code) {
-    if (mbar_test(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, c, status, code);
-}
-
 // Bounded wait by a converged warp; the answer is the same in every lane.
 __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, Ctrl* c, uint32_t* status, uint32_t code) {
     if (__all_sync(0xffffffffu, mbar_test(bar, parity))) return true;
@@ -231,30 +234,7 @@ __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src, ui
 // K-halves of an 8-row band are 128 bytes apart (leading byte offset) and bands are 256 bytes
 // apart (stride byte offset).  Offsets are stored >> 4; bit 46 is the descriptor version.
 // The start address sits in the low 14 bits, so adding (bytes >> 4) moves the descriptor.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr) {
-    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(128 >> 4) << 16) | ((uint64_t)(256 >> 4) << 32) |
-           (1ull << 46);
-}
-
-template <bool I8>
-__device__ __forceinline__ void mma_issue(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
-    if (I8)
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "setp.ne.b32 p, %4, 0;\n\t"
-            "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
-            ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(kIdescI8), "r"(accumulate)
-            : "memory");
-    else
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "setp.ne.b32 p, %4, 0;\n\t"
-            "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
-            ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(kIdescF8), "r"(accumulate)
-            : "memory");
-}
-
-// The same two instructions for a converged warp: every lane executes them and the predicate lets
+// MMA issue and commit for a converged warp: every lane executes them and the predicate lets
 // one through (`on` is non-zero in lane 0 only, and only if the step is to be issued), so there
 // is no branch.  Descriptors are passed as their low words; the high word is constant.
 constexpr uint32_t kDescHi = (256u >> 4) | (1u << 14);   // stride byte offset 256, descriptor version 1
@@ -287,11 +267,6 @@ __device__ __forceinline__ void mma_commit_if(uint32_t on, uint32_t bar_s) {
 }
 // low word of the operand descriptor of a block at shared address saddr (leading byte offset 128)
 __device__ __forceinline__ uint32_t desc_lo(uint32_t saddr) { return ((saddr & 0x3FFFFu) >> 4) | ((128u >> 4) << 16); }
-
-__device__ __forceinline__ void mma_commit(uint64_t* bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
-                 : "memory");
-}
 
 // 32 consecutive columns of this warp's 32 TMEM lanes: lane i receives row i, v[j] = column j.
 // The operands are declared read-write so that a landing buffer keeps its registers for the
@@ -332,16 +307,8 @@ __device__ __forceinline__ uint32_t lds32(uint32_t addr) {
     asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
     return v;
 }
-__device__ __forceinline__ uint4 lds128(uint32_t addr) {
-    uint4 v;
-    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
-    return v;
-}
 __device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) {
     asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
-}
-__device__ __forceinline__ void sts64(uint32_t addr, uint32_t x, uint32_t y) {
-    asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(addr), "r"(x), "r"(y) : "memory");
 }
 __device__ __forceinline__ void sts128(uint32_t addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
