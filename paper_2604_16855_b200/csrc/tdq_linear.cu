@@ -173,7 +173,12 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
 __device__ __forceinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, Ctrl* c, uint32_t* status, uint32_t code) {
     long long t0 = 0;
 #pragma unroll 1
-    while (!mbar_try(bar, parity)) {
+    for (;;) {
+        // a burst of sleeping waits between two looks at the abort flag and the clock: waiting warps
+        // share their scheduler with working ones, so the waiting loop is kept to a few instructions
+#pragma unroll 1
+        for (int i = 0; i < 32; ++i)
+            if (mbar_try(bar, parity)) return true;
         if (c->abort_flag) return false;
         const long long now = clock64();
         if (t0 == 0) t0 = now;
@@ -183,7 +188,6 @@ __device__ __forceinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, C
             return false;
         }
     }
-    return true;
 }
 
 // Bounded wait by a converged warp; the answer is the same in every lane.
