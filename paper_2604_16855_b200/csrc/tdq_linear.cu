@@ -84,7 +84,8 @@ constexpr int kThreads = (kPromoWarp0 + kPromoWarps) * 32;   // 640
 constexpr int kStripBytes = kCols * 4;   // one thread's 32 raw fp32 sums
 constexpr int kStagingBytes = kPromoWarps * 32 * kStripBytes;
 constexpr int kWsbBytes = kPromoWarps * 256;   // per warp: 32 output-channel scales and 32 biases
-constexpr int kCtrlBytes = 256;
+constexpr int kCtrlBytes = 384;
+constexpr int kMaxItemBufs = 4;          // copies of a work item's scales and resident A block in flight
 constexpr int kSmemLimit = 232448;       // 227 KB per CTA
 constexpr uint32_t kTmemCols = kSlots * kBN;
 constexpr long long kTimeoutCycles = 2000000000LL;
@@ -110,7 +111,9 @@ struct LinArgs {
     int32_t tiles_m, tiles_n, n_parts;
     int32_t a_resident;        // the item's whole A block stays in shared memory
     int32_t n_stages;
-    uint32_t ares_off, ring_off, stage_bytes, staging_off;   // shared-memory carve-up
+    uint32_t ring_off, stage_bytes, staging_off;   // shared-memory carve-up
+    uint32_t ibuf_bytes;       // one item buffer: the item's scales, then its A blocks if resident
+    int32_t n_ibuf;            // item buffers (1..kMaxItemBufs): the producer runs that many items ahead
     void* y;
     int64_t y_stride;
     int32_t* acc_debug;
@@ -127,7 +130,7 @@ struct LinArgs {
 struct Ctrl {
     uint64_t full[kMaxStages], empty[kMaxStages];
     uint64_t tfull[kSlots], tempty[kSlots];
-    uint64_t a_full, a_empty;
+    uint64_t a_full[kMaxItemBufs], a_empty[kMaxItemBufs];
     uint32_t tmem_base;
     volatile int abort_flag;
 };
@@ -428,8 +431,11 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
     extern __shared__ __align__(128) uint8_t smem_raw[];   // no static shared memory: the window starts aligned
     Ctrl* c = reinterpret_cast<Ctrl*>(smem_raw);
     const uint32_t sm_s = smem_u32(smem_raw);
-    const uint32_t scales_s = sm_s + kCtrlBytes;        // [Kg][128] floats of the item
-    const uint32_t ares_s = sm_s + a.ares_off;          // [n_steps] operand blocks of the item, if resident
+    // item buffer b: [Kg][128] floats of the item's scales, then its [n_steps] operand blocks if resident.
+    // Item number ic of this CTA uses buffer ic % n_ibuf; (ib, iu) below are that index and the parity of
+    // ic / n_ibuf, which is the phase of the buffer's two barriers.
+    const uint32_t ibuf_s = sm_s + kCtrlBytes;
+    const uint32_t a_in_ibuf = (uint32_t)a.Kg * kScaleBlock;
     const uint32_t ring_s = sm_s + a.ring_off;
     const int t = threadIdx.x, warp = t >> 5, lane = t & 31;
     const bool resident = a.a_resident != 0;
@@ -438,8 +444,10 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
         const uint32_t n_issuers = a.steps_per_grp <= 2 ? 2u : 1u;   // MMA-issuing warps
         for (int i = 0; i < kMaxStages; ++i) { mbar_init(&c->full[i], 1); mbar_init(&c->empty[i], n_issuers); }
         for (int i = 0; i < kSlots; ++i) { mbar_init(&c->tfull[i], 1); mbar_init(&c->tempty[i], kPromoWarps); }
-        mbar_init(&c->a_full, FUSED ? kPromoWarps : 1);
-        mbar_init(&c->a_empty, n_issuers + kPromoWarps);
+        for (int i = 0; i < kMaxItemBufs; ++i) {
+            mbar_init(&c->a_full[i], FUSED ? kPromoWarps : 1);
+            mbar_init(&c->a_empty[i], n_issuers + kPromoWarps);
+        }
         c->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -465,29 +473,32 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
         // warp-mates sit at the final barrier was measured to execute several times slower.
         if (warp < kProdWarps) {
             // ------------------------------------------------------------ producers (lane 0 issues)
-            uint32_t sc = 0, s = 0, ph = 0, ic = 0;   // stage counter, its ring slot and phase; items so far
+            uint32_t sc = 0, s = 0, ph = 0;   // stage counter, its ring slot and phase
+            uint32_t ib = 0, iu = 0;          // item buffer and its phase
             bool ok = true;
-            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++ic) {
+            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
                 const int mt = item / a.n_parts, part = item % a.n_parts;
                 const uint8_t* a_src = a.a_blocks + (int64_t)mt * a.n_steps * kBlock;
                 if (warp == 0 && !FUSED) {
-                    ok = mbar_wait_warp(&c->a_empty, (ic & 1) ^ 1, c, a.status, 1u);
+                    ok = mbar_wait_warp(&c->a_empty[ib], iu ^ 1, c, a.status, 1u);
                     if (!ok) break;
                     if (lane == 0) {
                     const uint32_t sbytes = (uint32_t)a.Kg * kScaleBlock;
-                    mbar_expect_tx(&c->a_full, sbytes + (resident ? (uint32_t)a.n_steps * kBlock : 0u));
+                    const uint32_t scales_s = ibuf_s + ib * a.ibuf_bytes, ares_s = scales_s + a_in_ibuf;
+                    mbar_expect_tx(&c->a_full[ib], sbytes + (resident ? (uint32_t)a.n_steps * kBlock : 0u));
                     const uint8_t* s_src = a.s_blocks + (int64_t)mt * a.Kg * kScaleBlock;
                     for (uint32_t off = 0; off < sbytes; off += 16384u)
-                        bulk_load(scales_s + off, s_src + off, min(16384u, sbytes - off), &c->a_full);
+                        bulk_load(scales_s + off, s_src + off, min(16384u, sbytes - off), &c->a_full[ib]);
                     if (resident)
                         for (int kc = 0; kc < n_chunks; ++kc) {
                             const int nk = min(kChunk, a.n_steps - kc * kChunk);
                             bulk_load(ares_s + kc * kChunk * kBlock, a_src + (int64_t)kc * kChunk * kBlock,
-                                      (uint32_t)nk * kBlock, &c->a_full);
+                                      (uint32_t)nk * kBlock, &c->a_full[ib]);
                         }
                     }
                     __syncwarp();
                 }
+                if (++ib == (uint32_t)a.n_ibuf) { ib = 0; iu ^= 1; }
                 for (int nt = part_begin(part); nt < part_begin(part + 1) && ok; ++nt) {
                     const uint8_t* b_src = a.b_blocks + (int64_t)nt * a.n_steps * kBlock;
                     for (int kc = 0; kc < n_chunks; ++kc, ++sc) {
@@ -518,7 +529,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
             // groups' time for its bookkeeping; wider groups chain into one slot and stay with one warp.
             const uint32_t me = (uint32_t)(warp - kMmaWarp);
             const uint32_t lane0 = lane == 0 ? 1u : 0u;
-            const uint32_t ares_lo = desc_lo(ares_s), ring_lo = desc_lo(ring_s);
+            const uint32_t ring_lo = desc_lo(ring_s);
             const uint32_t stage_step = a.stage_bytes >> 4, n_stages = (uint32_t)a.n_stages;
             const uint32_t a_in_stage = resident ? 0u : (uint32_t)(kChunk * (kBlock >> 4));
             const uint32_t empty_s = smem_u32(&c->empty[0]), tfull_s = smem_u32(&c->tfull[0]);
@@ -532,7 +543,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
             auto role = [&](auto mode_tag) {
                 constexpr int MODE = decltype(mode_tag)::value;
                 constexpr bool DUAL = MODE == 0, QUAD = MODE == 1, DUAL2 = MODE == 3;
-                uint32_t s = 0, ph = 0, ic = 0;
+                uint32_t s = 0, ph = 0, ib = 0, iu = 0;
                 bool ok = true;
                 // DUAL: this warp's two slots (me and me + 2), everything about them precomputed
                 const uint32_t tm_a = tmem_base + me * kBN, tm_b = tm_a + 2 * kBN;
@@ -542,10 +553,11 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                 uint32_t q_a = 1, q_b = 1;     // parity to wait for on tempty of each slot; a fresh barrier passes parity 1
                 // otherwise: one slot at a time
                 uint32_t qm = 0xFu;            // the same parities as a mask, bit = slot
-                for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++ic) {
+                for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
                     const int part = item % a.n_parts;
                     const int n_tiles = part_begin(part + 1) - part_begin(part);
-                    ok = mbar_wait_warp(&c->a_full, ic & 1, c, a.status, 6u);
+                    ok = mbar_wait_warp(&c->a_full[ib], iu, c, a.status, 6u);
+                    const uint32_t ares_lo = desc_lo(ibuf_s + ib * a.ibuf_bytes + a_in_ibuf);
                     for (int tl = 0; tl < n_tiles && ok; ++tl) {
                         int sub = 0;
                         uint32_t slot = 0;
@@ -639,7 +651,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                             if (++s == n_stages) { s = 0; ph ^= 1; }
                         }
                     }
-                    if (ok) mma_commit_if(lane0, smem_u32(&c->a_empty));
+                    if (ok) mma_commit_if(lane0, smem_u32(&c->a_empty[ib]));
+                    if (++ib == (uint32_t)a.n_ibuf) { ib = 0; iu ^= 1; }
                 }
             };
             if (spg == 1) role(std::integral_constant<int, 0>{});
@@ -668,7 +681,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
         const uint32_t strip_row = strip_w + (uint32_t)lane * kRowBytes;
         const uint32_t swz = YBF16 ? (((uint32_t)lane >> 1) & 3u) : ((uint32_t)lane & 7u);   // chunk c sits at c ^ swz
         const uint32_t wsb_s = strips_s + kStagingBytes + (uint32_t)pw * 256;
-        const uint32_t my_scale_s = scales_s + (uint32_t)row * 4;
+        uint32_t ib = 0, iu = 0;                      // item buffer and its phase
+        uint32_t my_scale_s = ibuf_s + (uint32_t)row * 4;   // this row's scales in the current item buffer
 
         uint64_t yacc[kCols / 2];      // 32 floats of one output row, packed in pairs
         uint32_t v[kCols];             // landing buffer: this thread's 32 columns of a slot
@@ -688,12 +702,14 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
             nt_end = part_begin(part + 1);
             m = (int64_t)mt * kBM + row;
             row_ok = m < a.M;
+            const uint32_t scales_s = ibuf_s + ib * a.ibuf_bytes, ares_s = scales_s + a_in_ibuf;
+            my_scale_s = scales_s + (uint32_t)row * 4;
             if (FUSED) {
                 // The previous item's A and scales are free once every MMA that read them has completed and
                 // every promotion warp has left the item (a_empty counts both).  Then thread = (row, group
                 // mod 4) quantizes its groups: Algorithm S1 steps 2-7 in registers, codes expanded to operand
                 // bytes in the block's core-matrix order, the step to the scale block.
-                ok = mbar_wait_warp(&c->a_empty, (ic & 1) ^ 1, c, a.status, 1u);
+                ok = mbar_wait_warp(&c->a_empty[ib], iu ^ 1, c, a.status, 1u);
                 if (ok) {
                     constexpr bool XBF = FUSED == 1;
                     const int pt = pw * 32 + lane, r = pt & (kBM - 1);
@@ -720,10 +736,10 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                     // written through the generic proxy, read by the tensor core through the async proxy
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
-                    mbar_arrive_lane0(&c->a_full, lane);
+                    mbar_arrive_lane0(&c->a_full[ib], lane);
                 }
             }
-            if (ok) ok = mbar_wait_warp(&c->a_full, ic & 1, c, a.status, 7u);
+            if (ok) ok = mbar_wait_warp(&c->a_full[ib], iu, c, a.status, 7u);
         };
         auto begin_tile = [&]() {
             n0 = (int64_t)nt * kBN + col0;
@@ -808,9 +824,9 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                 // overwrite them through the async proxy, which only a proxy fence orders after the reads
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
-                mbar_arrive_lane0(&c->a_empty, lane);
+                mbar_arrive_lane0(&c->a_empty[ib], lane);
+                if (++ib == (uint32_t)a.n_ibuf) { ib = 0; iu ^= 1; }
                 item += gridDim.x;
-                ++ic;
                 if (item < n_items) begin_item();
             }
             if (ok && item < n_items) begin_tile();
@@ -946,7 +962,8 @@ bool encode_y_map(CUtensorMap* map, void* y, bool bf16, int64_t M, int64_t O, in
 struct Plan {
     int64_t tiles_m, tiles_n;
     int32_t n_steps, n_chunks, Kg, n_parts, a_resident, n_stages;
-    uint32_t ares_off, ring_off, stage_bytes, staging_off, smem_bytes;
+    uint32_t ring_off, stage_bytes, staging_off, smem_bytes, ibuf_bytes;
+    int32_t n_ibuf;
     size_t a_bytes, b_bytes, s_bytes;   // operand and scale blocks in the workspace
 };
 
@@ -969,20 +986,26 @@ bool make_plan(int64_t M, int64_t I_pad, int64_t O, int32_t g, int n_sm, Plan& p
     const int64_t a_res = (int64_t)p.n_steps * kBlock;
     const int64_t stage_b = (int64_t)kChunk * kBlock, stage_ab = 2 * stage_b;
     const int64_t stages_res = (kSmemLimit - fixed - a_res) / stage_b;
-    p.ares_off = (uint32_t)(kCtrlBytes + scales);
     if (stages_res >= 3) {
         p.a_resident = 1;
-        p.n_stages = (int32_t)(stages_res > kMaxStages ? kMaxStages : stages_res);
+        p.ibuf_bytes = (uint32_t)(scales + a_res);
+        // further item buffers while at least six stages remain: with short contractions the hand-over
+        // between work items, not the ring, is what the tensor core waits for
+        p.n_ibuf = 1;
+        while (p.n_ibuf < kMaxItemBufs && (kSmemLimit - fixed - a_res - (int64_t)p.n_ibuf * p.ibuf_bytes) / stage_b >= 6) ++p.n_ibuf;
+        const int64_t st = (kSmemLimit - fixed - a_res - (int64_t)(p.n_ibuf - 1) * p.ibuf_bytes) / stage_b;
+        p.n_stages = (int32_t)(st > kMaxStages ? kMaxStages : st);
         p.stage_bytes = (uint32_t)stage_b;
-        p.ring_off = p.ares_off + (uint32_t)a_res;
     } else {
         const int64_t st = (kSmemLimit - fixed) / stage_ab;
         if (st < 2) return false;
         p.a_resident = 0;
+        p.ibuf_bytes = (uint32_t)scales;
+        p.n_ibuf = 1;
         p.n_stages = (int32_t)(st > kMaxStages ? kMaxStages : st);
         p.stage_bytes = (uint32_t)stage_ab;
-        p.ring_off = p.ares_off;
     }
+    p.ring_off = (uint32_t)kCtrlBytes + (uint32_t)p.n_ibuf * p.ibuf_bytes;
     p.staging_off = p.ring_off + (uint32_t)p.n_stages * p.stage_bytes;
     p.smem_bytes = p.staging_off + 1024 + kStagingBytes + kWsbBytes;
     // split the column tiles of a row block into parts so that the items fill the SMs evenly
@@ -1072,7 +1095,8 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
     a.n_steps = p.n_steps; a.steps_per_grp = e.steps_per_grp; a.Kg = p.Kg;
     a.tiles_m = (int32_t)p.tiles_m; a.tiles_n = e.tiles_n; a.n_parts = p.n_parts;
     a.a_resident = p.a_resident; a.n_stages = p.n_stages;
-    a.ares_off = p.ares_off; a.ring_off = p.ring_off; a.stage_bytes = p.stage_bytes;
+    a.ring_off = p.ring_off; a.stage_bytes = p.stage_bytes;
+    a.ibuf_bytes = p.ibuf_bytes; a.n_ibuf = p.n_ibuf;
     a.staging_off = p.staging_off;
     a.y = y; a.y_stride = y_row_stride; a.acc_debug = acc_debug;
     a.status = reinterpret_cast<uint32_t*>(workspace);
