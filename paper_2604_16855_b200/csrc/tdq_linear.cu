@@ -120,6 +120,11 @@ struct LinArgs {
     uint32_t* status;
     int32_t tma_ok;            // y can be written with bulk tensor stores (16-byte aligned base and row pitch)
     float out_scale;           // 2^18 (E4M3 route) or 2^-8 (int8 route)
+    // resident A without the fused producer: the promotion warps unpack the item's codes themselves
+    const uint8_t* xcodes;
+    const float* xscale;
+    int32_t row_bytes;         // I_pad / 2
+    int32_t unpack_a;
     // fused producer only: the activations themselves and the quantizer's parameters
     const void* x;
     int64_t x_stride;          // elements between rows of x
@@ -445,7 +450,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
         for (int i = 0; i < kMaxStages; ++i) { mbar_init(&c->full[i], 1); mbar_init(&c->empty[i], n_issuers); }
         for (int i = 0; i < kSlots; ++i) { mbar_init(&c->tfull[i], 1); mbar_init(&c->tempty[i], kPromoWarps); }
         for (int i = 0; i < kMaxItemBufs; ++i) {
-            mbar_init(&c->a_full[i], FUSED ? kPromoWarps : 1);
+            mbar_init(&c->a_full[i], (FUSED || a.unpack_a) ? kPromoWarps : 1);
             mbar_init(&c->a_empty[i], n_issuers + kPromoWarps);
         }
         c->abort_flag = 0;
@@ -479,7 +484,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
             for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
                 const int mt = item / a.n_parts, part = item % a.n_parts;
                 const uint8_t* a_src = a.a_blocks + (int64_t)mt * a.n_steps * kBlock;
-                if (warp == 0 && !FUSED) {
+                if (warp == 0 && !FUSED && !a.unpack_a) {
                     ok = mbar_wait_warp(&c->a_empty[ib], iu ^ 1, c, a.status, 1u);
                     if (!ok) break;
                     if (lane == 0) {
@@ -734,6 +739,41 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                         sts32(scales_s + (uint32_t)k * kScaleBlock + (uint32_t)r * 4, __float_as_uint(delta));
                     }
                     // written through the generic proxy, read by the tensor core through the async proxy
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    mbar_arrive_lane0(&c->a_full[ib], lane);
+                }
+            }
+            if (!FUSED && a.unpack_a) {
+                // Packed codes -> operand bytes, straight into the item buffer (no pass through global
+                // memory): thread pt takes row pt / 4 and every fourth K-step from pt % 4, so that a warp
+                // reads 64 contiguous bytes of each of 8 rows.
+                ok = mbar_wait_warp(&c->a_empty[ib], iu ^ 1, c, a.status, 1u);
+                if (ok) {
+                    const int pt = pw * 32 + lane, r = pt >> 2;
+                    const int64_t mr = (int64_t)mt * kBM + r;
+                    const uint32_t off = (uint32_t)((r >> 3) * 256 + (r & 7) * 16);
+                    const uint8_t* src = a.xcodes + mr * a.row_bytes;
+#pragma unroll 1
+                    for (int ks = pt & 3; ks < a.n_steps; ks += 4) {
+                        uint4 p4 = make_uint4(0u, 0u, 0u, 0u);
+                        if (mr < a.M) p4 = __ldg(reinterpret_cast<const uint4*>(src + ks * 16));
+                        uint4 c0, c1;
+                        expand8<I8>(p4.x, c0.x, c0.y);
+                        expand8<I8>(p4.y, c0.z, c0.w);
+                        expand8<I8>(p4.z, c1.x, c1.y);
+                        expand8<I8>(p4.w, c1.z, c1.w);
+                        const uint32_t dst = ares_s + (uint32_t)ks * kBlock + off;
+                        sts128(dst, c0.x, c0.y, c0.z, c0.w);
+                        sts128(dst + 128, c1.x, c1.y, c1.z, c1.w);
+                    }
+                    // scales: [group][128 rows]; thread pt takes row pt % 128 and every fourth group
+                    const int rs = pt & (kBM - 1);
+                    const int64_t ms = (int64_t)mt * kBM + rs;
+#pragma unroll 1
+                    for (int k = pt >> 7; k < a.Kg; k += kPromoWarps * 32 / kBM)
+                        sts32(scales_s + (uint32_t)k * kScaleBlock + (uint32_t)rs * 4,
+                              ms < a.M ? __float_as_uint(__ldg(a.xscale + ms * a.Kg + k)) : 0u);
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
                     mbar_arrive_lane0(&c->a_full[ib], lane);
@@ -1085,7 +1125,12 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
     e.n_steps = p.n_steps; e.n_chunks = p.n_chunks;
     e.steps_per_grp = group_size / 32;
     e.Kg = p.Kg;
-    e.tiles_m = fx ? 0 : (int32_t)p.tiles_m;   // fused: only the weights are expanded
+    // The kernel can unpack a resident A block itself, which saves the pass that writes A blocks to the
+    // workspace; its promotion warps do that at the start of an item, though, with the tensor core idle,
+    // so it only pays when an item carries much more work than its own unpacking.
+    const int64_t steps_per_item = (p.tiles_n + p.n_parts - 1) / p.n_parts * (int64_t)p.n_steps;
+    const bool unpack_a = !fx && p.a_resident && steps_per_item >= 256;
+    e.tiles_m = (fx || unpack_a) ? 0 : (int32_t)p.tiles_m;   // then only the weights are expanded here
     e.tiles_n = (int32_t)p.tiles_n;
 
     LinArgs a;
@@ -1109,6 +1154,7 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
         encode_y_map(&ymap, y, y_dtype == TDQ_BF16, M, O, y_row_stride))
         a.tma_ok = 1;
     a.out_scale = i8 ? 0.00390625f : 262144.0f;
+    a.xcodes = xcodes; a.xscale = xscale; a.row_bytes = e.row_bytes; a.unpack_a = unpack_a ? 1 : 0;
     a.x = fx ? fx->x : nullptr;
     a.x_stride = fx ? fx->row_stride : 0;
     a.seven_tau = fx ? fx->seven_tau : 0.0f;
