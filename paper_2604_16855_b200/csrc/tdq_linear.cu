@@ -296,6 +296,17 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* v) {
         : "memory");
 }
 
+// the same for 16 columns
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* v) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]),
+          "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15])
+        : "r"(taddr)
+        : "memory");
+}
+
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -690,23 +701,24 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
         uint32_t my_scale_s = ibuf_s + (uint32_t)row * 4;   // this row's scales in the current item buffer
 
         uint64_t yacc[kCols / 2];      // 32 floats of one output row, packed in pairs
-        uint32_t v[kCols];             // landing buffer: this thread's 32 columns of a slot
+        // landing buffer: this thread's 32 columns of a slot; 16 at a time in the fused kernel, whose
+        // quantizer code leaves the promotion loop fewer registers
+        constexpr int kLand = FUSED ? kCols / 2 : kCols;
+        uint32_t v[kLand];
 #pragma unroll
-        for (int q = 0; q < kCols; ++q) v[q] = 0u;
+        for (int q = 0; q < kLand; ++q) v[q] = 0u;
         uint32_t ic = 0;                 // items so far
         uint32_t p_full[kSlots] = {0u, 0u, 0u, 0u};   // parity of the completion of tfull[s] to wait for next
         int item = blockIdx.x, mt = 0, nt = 0, nt_end = 0;
-        int64_t m = 0, n0 = 0;
+        int64_t n0 = 0;
         float w0 = 0.f, b0 = 0.f;        // channel scale and bias of column n0 + lane
-        bool ok = true, row_ok = false;
+        bool ok = true;
 
         auto begin_item = [&]() {
             mt = item / a.n_parts;
             const int part = item % a.n_parts;
             nt = part_begin(part);
             nt_end = part_begin(part + 1);
-            m = (int64_t)mt * kBM + row;
-            row_ok = m < a.M;
             const uint32_t scales_s = ibuf_s + ib * a.ibuf_bytes, ares_s = scales_s + a_in_ibuf;
             my_scale_s = scales_s + (uint32_t)row * 4;
             if (FUSED) {
@@ -884,26 +896,34 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
             if (!__all_sync(0xffffffffu, ready)) ok = mbar_wait_warp(&c->tfull[U], p_full[U], c, a.status, 2u);
             p_full[U] ^= 1u;
             tc_fence_after();
-            tmem_ld32(tmem_row_r + U * kBN, v);
+            if (FUSED) tmem_ld16(tmem_row_r + U * kBN, v);
+            else tmem_ld32(tmem_row_r + U * kBN, v);
         };
         auto consume = [&](auto u_tag, uint32_t scale_q, int k) -> bool {
             constexpr uint32_t U = decltype(u_tag)::value, N = (U + 1) & (kSlots - 1);
             const uint32_t dbits = lds32(scale_q + U * kScaleBlock);
             const uint64_t d2 = pack2(dbits, dbits);
             const bool next_ready = mbar_test_s(tfull_s + N * 8, p_full[N]);
-            tmem_ld_wait();                               // v has landed: the slot is drained
-            tc_fence_before();
+            tmem_ld_wait();                               // v has landed
+            if (FUSED) {                                  // first half folded in, then the second half takes its place
+#pragma unroll
+                for (int q = 0; q < kLand / 2; ++q) fma2(yacc[q], pack2(v[2 * q], v[2 * q + 1]), d2);
+                tmem_ld16(tmem_row_r + U * kBN + kLand, v);
+                tmem_ld_wait();
+            }
+            tc_fence_before();                            // the slot is drained
             __syncwarp();
             mbar_arrive_lane0_s(tempty_s + U * 8, lane);
             if (DBG) {
-                if (a.acc_debug && row_ok) debug_store<I8>(a, v, m, n0, k + (int)U);
+                const int64_t m = (int64_t)mt * kBM + row;
+                if (a.acc_debug && m < a.M) debug_store<I8>(a, v, m, n0, k + (int)U);
             }
             if (I8) {
 #pragma unroll
-                for (int q = 0; q < kCols; ++q) v[q] = __float_as_uint((float)(int32_t)v[q]);
+                for (int q = 0; q < kLand; ++q) v[q] = __float_as_uint((float)(int32_t)v[q]);
             }
 #pragma unroll
-            for (int q = 0; q < kCols / 2; ++q) fma2(yacc[q], pack2(v[2 * q], v[2 * q + 1]), d2);
+            for (int q = 0; q < kLand / 2; ++q) fma2(yacc[(FUSED ? kLand / 2 : 0) + q], pack2(v[2 * q], v[2 * q + 1]), d2);
             return next_ready;
         };
         const std::integral_constant<uint32_t, 0> u0{};
