@@ -422,7 +422,17 @@ def run_tdq(args):
 
     total_ms, q_ms, l_ms, e2e_ms = max_over_ranks([total_ms, q_ms, l_ms, e2e_ms], dev, world)
     fused = sweep = None
+    q_iso_ms = l_iso_ms = None
     if world == 1 and not args.no_extras:
+        # each kernel on its own, launched back to back from a graph over rotating buffers: no other
+        # kernel and no event node between two launches (the in-step figures above include those gaps)
+        n_iso = max(nsets, int(np.ceil(2.5 * L2_BYTES / (M * C * esize))))
+        xi = xs + [xs[0].clone() for _ in range(n_iso - nsets)]
+        q_iso_ms = time_graph(lambda i: tdq.quantize_act(xi[i % n_iso], params, codes=codes[i % nsets], scale=scales[i % nsets]),
+                              4 * n_iso)
+        del xi
+        l_iso_ms = time_graph(lambda i: tdq.w4a4_linear(codes[i % nsets], scales[i % nsets], wcodes, wscale, y=ys[i % nsets],
+                                                        workspace=wsp), 8 * nsets)
         fused = fused_leg(tdq, xs, wcodes, wscale, ys, wsp, M, C, O, esize)
         del xs, codes, scales, ys
         torch.cuda.empty_cache()
@@ -439,10 +449,16 @@ def run_tdq(args):
         int8_peak = 2.0 * peaks["bf16_tflops"]            # nominal int8 : bf16 ratio on the measured bf16 peak
         q_kernel = dict(name="tdq_quantize_act", ms=q_ms / K, gbs=q_gbs, frac_hbm=q_gbs / peaks["hbm_gbs"],
                         frac_hbm_8tbs=q_gbs / 8000.0, algorithmic_bytes=qb)
+        if q_iso_ms:
+            q_kernel.update(back_to_back_ms=q_iso_ms, back_to_back_gbs=qb / (q_iso_ms * 1e-3) / 1e9,
+                            back_to_back_frac_hbm=qb / (q_iso_ms * 1e-3) / 1e9 / peaks["hbm_gbs"])
         l_kernel = dict(name="tdq_w4a4_linear", ms=l_ms / K, tops=l_tops, frac_int8=l_tops / int8_peak,
                         frac_int8_4500=l_tops / 4500.0, gbs=l_gbs, frac_hbm=l_gbs / peaks["hbm_gbs"],
                         algorithmic_bytes=lb, ops=ops,
                         bound="hbm" if lb / peaks["hbm_gbs"] / 1e9 > ops / int8_peak / 1e12 else "tensor")
+        if l_iso_ms:
+            l_kernel.update(back_to_back_ms=l_iso_ms, back_to_back_tops=ops / (l_iso_ms * 1e-3) / 1e12,
+                            back_to_back_gbs=lb / (l_iso_ms * 1e-3) / 1e9)
         if l_ms >= q_ms:
             if l_kernel["bound"] == "hbm":
                 roof = dict(kernel="tdq_w4a4_linear", bound="hbm", achieved=l_gbs, peak=peaks["hbm_gbs"],
