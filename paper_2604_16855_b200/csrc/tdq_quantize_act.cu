@@ -1,7 +1,12 @@
 // tdq_quantize_act: token-group dual-constraint activation quantizer (Algorithm S1 steps 1-7).
 //
-// Two kernels:
-//   * act_g32_kernel   g = 32, C % 32 == 0, 16-byte aligned rows.  A CTA stages a tile of
+// Three kernels:
+//   * act_g32_ring_kernel   the fast path on dense rows (row stride == C): persistent, two CTAs per
+//     SM; one producer lane streams 16 KB tiles of 256 groups into a shared-memory ring with 1-D
+//     bulk copies and mbarrier transaction counts, eight consumer warps take one group per thread
+//     (the per-group arithmetic is in tdq_act_group.cuh).
+//   * act_g32_kernel   the same per-group code for strided rows: g = 32, C % 32 == 0, 16-byte
+//     aligned rows.  A CTA stages a tile of
 //     consecutive token-groups in shared memory with coalesced 128-bit loads (XOR-swizzled
 //     so the read-back is conflict free); then every thread owns one whole group in
 //     registers: max, sums, a pruned sorting network for the rank-k magnitude, the DCRP

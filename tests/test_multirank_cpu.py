@@ -47,3 +47,12 @@ def test_two_ranks_take_the_slowest_time_and_sum_the_work():
         assert p.exitcode == 0
     assert got == [11.0, 3.0, 7.0]
     assert abs(rate - 2 * 1000.0 / 11e-3) < 1e-6
+
+
+def test_graph_steps_divides_the_step_count_and_respects_the_buffer_rotation():
+    import bench
+    for K, nsets in [(1000, 2), (50, 2), (7, 2), (64, 3), (97, 2), (128, 4), (3, 2)]:
+        G = bench.graph_steps(K, nsets)
+        assert K % G == 0 and 1 <= G <= max(K, 64)
+        # either a whole number of rotations per graph, or one graph that holds every step
+        assert G % nsets == 0 or G == K
