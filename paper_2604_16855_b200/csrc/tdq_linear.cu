@@ -392,12 +392,14 @@ struct ExpandArgs {
     int32_t row_bytes;       // I_pad / 2
     int32_t n_steps, n_chunks, steps_per_grp, Kg;
     int32_t tiles_m, tiles_n;
+    uint32_t* status;        // the workspace's status words, cleared here for the GEMM that follows
 };
 
 // One CTA rewrites one (128-row block, 4 K-steps) piece: thread t takes row t / 4 and K-step t % 4.
 template <bool I8>
 __global__ void __launch_bounds__(kExpandThreads) expand_kernel(ExpandArgs a) {
     const int piece = blockIdx.x;
+    if (piece == 0 && threadIdx.x < 4) a.status[threadIdx.x] = 0u;   // saves a separate memset in front of every call
     const int blk = piece / a.n_chunks, kc = piece % a.n_chunks;
     const int r = threadIdx.x >> 2;
     const int ks = kc * kChunk + (threadIdx.x & 3);
@@ -1152,6 +1154,7 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
     const bool unpack_a = !fx && p.a_resident && steps_per_item >= 256;
     e.tiles_m = (fx || unpack_a) ? 0 : (int32_t)p.tiles_m;   // then only the weights are expanded here
     e.tiles_n = (int32_t)p.tiles_n;
+    e.status = reinterpret_cast<uint32_t*>(workspace);
 
     LinArgs a;
     a.a_blocks = e.a_blocks; a.b_blocks = e.b_blocks; a.s_blocks = e.s_blocks;
@@ -1192,7 +1195,6 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
     }
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess)
         return TDQ_ERR_CUDA;
-    if (cudaMemsetAsync(workspace, 0, 16, stream) != cudaSuccess) return TDQ_ERR_CUDA;
 
     const unsigned pieces = (unsigned)((e.tiles_m + e.tiles_n) * p.n_chunks);
     if (i8)
