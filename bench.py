@@ -423,6 +423,7 @@ def run_tdq(args):
     total_ms, q_ms, l_ms, e2e_ms = max_over_ranks([total_ms, q_ms, l_ms, e2e_ms], dev, world)
     fused = sweep = None
     q_iso_ms = l_iso_ms = None
+    q_switch_ms = None
     if world == 1 and not args.no_extras:
         # each kernel on its own, launched back to back from a graph over rotating buffers: no other
         # kernel and no event node between two launches (the in-step figures above include those gaps)
@@ -430,6 +431,13 @@ def run_tdq(args):
         xi = xs + [xs[0].clone() for _ in range(n_iso - nsets)]
         q_iso_ms = time_graph(lambda i: tdq.quantize_act(xi[i % n_iso], params, codes=codes[i % nsets], scale=scales[i % nsets]),
                               4 * n_iso)
+        # the quantizer with one or both bounds switched off (the paper's C1-only, C2-only and
+        # DSTG-only ablation settings), back to back like the line above
+        q_switch_ms = {}
+        for label, flags in (("c1_only", tdq.ENABLE_C1), ("c2_only", tdq.ENABLE_C2), ("dstg_only", 0)):
+            pf = tdq.act_params(flags=flags)
+            q_switch_ms[label] = time_graph(lambda i: tdq.quantize_act(xi[i % n_iso], pf, codes=codes[i % nsets],
+                                                                       scale=scales[i % nsets]), 4 * n_iso)
         del xi
         l_iso_ms = time_graph(lambda i: tdq.w4a4_linear(codes[i % nsets], scales[i % nsets], wcodes, wscale, y=ys[i % nsets],
                                                         workspace=wsp), 8 * nsets)
@@ -452,6 +460,7 @@ def run_tdq(args):
         if q_iso_ms:
             q_kernel.update(back_to_back_ms=q_iso_ms, back_to_back_gbs=qb / (q_iso_ms * 1e-3) / 1e9,
                             back_to_back_frac_hbm=qb / (q_iso_ms * 1e-3) / 1e9 / peaks["hbm_gbs"])
+            q_kernel["back_to_back_ms_by_setting"] = q_switch_ms
         l_kernel = dict(name="tdq_w4a4_linear", ms=l_ms / K, tops=l_tops, frac_int8=l_tops / int8_peak,
                         frac_int8_4500=l_tops / 4500.0, gbs=l_gbs, frac_hbm=l_gbs / peaks["hbm_gbs"],
                         algorithmic_bytes=lb, ops=ops,
