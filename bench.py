@@ -424,6 +424,7 @@ def run_tdq(args):
     fused = sweep = None
     q_iso_ms = l_iso_ms = None
     q_switch_ms = None
+    q_nchw = None
     if world == 1 and not args.no_extras:
         # each kernel on its own, launched back to back from a graph over rotating buffers: no other
         # kernel and no event node between two launches (the in-step figures above include those gaps)
@@ -439,6 +440,16 @@ def run_tdq(args):
             q_switch_ms[label] = time_graph(lambda i: tdq.quantize_act(xi[i % n_iso], pf, codes=codes[i % nsets],
                                                                        scale=scales[i % nsets]), 4 * n_iso)
         del xi
+        # channel-major input of the same volume: a [B, C, 24, 24] feature map quantized along C in place
+        fm = [torch.randn((32, C, 24, 24), device=dev).mul_(torch.randn((32, 1, 24, 24), device=dev).exp_())
+              .to(torch.bfloat16 if case.x_is_bf16 else torch.float32) for _ in range(n_iso)]
+        Mf = 32 * 24 * 24
+        fcodes = torch.empty((Mf, C // 2), dtype=torch.uint8, device=dev)
+        fscale = torch.empty((Mf, C // 32), dtype=torch.float32, device=dev)
+        q_nchw_ms = time_graph(lambda i: tdq.quantize_act_nchw(fm[i % n_iso], params, codes=fcodes, scale=fscale), 4 * n_iso)
+        q_nchw = dict(name="tdq_quantize_act_nchw", x=[32, C, 24, 24], ms=q_nchw_ms,
+                      gbs=quant_bytes(Mf, C, esize) / (q_nchw_ms * 1e-3) / 1e9)
+        del fm, fcodes, fscale
         l_iso_ms = time_graph(lambda i: tdq.w4a4_linear(codes[i % nsets], scales[i % nsets], wcodes, wscale, y=ys[i % nsets],
                                                         workspace=wsp), 8 * nsets)
         fused = fused_leg(tdq, xs, wcodes, wscale, ys, wsp, M, C, O, esize)
@@ -490,7 +501,7 @@ def run_tdq(args):
                                cache="rotating %d buffer sets, %.0f MB per step (L2 is 126 MB)" % (nsets, step_bytes / 1e6),
                                launch=("CUDA graph of %d steps, replayed %d times" % (G, args.steps // G)) if G else "eager",
                                parallelism="rows sharded, %d replica(s)" % world),
-                   kernels=dict(quantize_act=q_kernel, w4a4_linear=l_kernel, fused=fused, sweep_cfg5=sweep,
+                   kernels=dict(quantize_act=q_kernel, quantize_act_nchw=q_nchw, w4a4_linear=l_kernel, fused=fused, sweep_cfg5=sweep,
                                 step_tokens_per_s=world * M * K / (total_ms * 1e-3)),
                    roofline=roof, clocks=clocks, gpu_launches=int(launches),
                    e2e=dict(value=e2e_value, unit="GB/s", ms_per_step=e2e_ms / e2e_steps,

@@ -83,6 +83,22 @@ tdq_status tdq_quantize_act(const void* x, tdq_dtype x_dtype, int64_t B, int64_t
                             uint8_t* codes, float* scale, float* offset, void* cuda_stream);
 
 /*
+ * The same quantizer for channel-major input (the 4-D branch of Supp. S1.1, where a feature
+ * map [B, C, H, W] is quantized along C): x is read in place, without the permuted copy that
+ * tdq_quantize_act would need, and the outputs are token-major like tdq_quantize_act's with
+ * token index (b*H + h)*W + w:   codes [B*H*W, C/2],  scale [B*H*W, C/32],  offset NULL or
+ * [B*H*W, C/32].  They can go straight into tdq_w4a4_linear (a 1x1 convolution).
+ *   x   [B, C, H, W] contiguous.  16-byte aligned x with H*W*sizeof(element) % 16 == 0 is read
+ *       with vector loads, anything else element by element.
+ * Fast path only: TDQ_ERR_UNSUPPORTED unless group_size == 32, C % 32 == 0, base_percentile
+ * gives the maximum (rank 32), codes is 16-byte aligned and, with C2 on, ceil(32 zr) is one
+ * of 4, 7, 10, 13, 16, 32; also if C/32 or B exceeds 65535.  Other errors as above.
+ */
+tdq_status tdq_quantize_act_nchw(const void* x, tdq_dtype x_dtype, int64_t B, int64_t C, int64_t H,
+                                 int64_t W, const tdq_act_params* p /* HOST */, uint8_t* codes,
+                                 float* scale, float* offset, void* cuda_stream);
+
+/*
  * Static weight quantizer, Eq. 4 with absmax per-output-channel scales:
  *   s_o = max(max_i |W[o,i]| / 7, 1e-8);  Q = clip(round_half_even(W / s_o), -8, 7).
  *   w       [O, I] row-major, contiguous, w_dtype.

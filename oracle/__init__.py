@@ -106,6 +106,17 @@ def quantize_act(x, g=32, tau=1.0, zr=0.2, p=1.0, flags=ENABLE_C1 | ENABLE_C2, C
     return out
 
 
+def quantize_act_nchw(x, **kw):
+    """The 4-D branch of Supp. S1.1: a feature map [B, C, H, W] is laid out as tokens [B, H*W, C] (a plain
+    transpose), then quantized along C by quantize_act.  Outputs are token-major: [B*H*W, ...]."""
+    x = np.asarray(x)
+    if x.ndim != 4:
+        raise ValueError("x must be [B, C, H, W]")
+    B, C, H, W = x.shape
+    tokens = np.ascontiguousarray(np.transpose(x, (0, 2, 3, 1))).reshape(B * H * W, C)
+    return quantize_act(tokens, **kw)
+
+
 def quantize_weight(w, pad_to=32):
     """Eq. 4 with absmax scales. Returns dict q int8 [O, I_pad], codes uint8, scale float32 [O]."""
     w, dt = _as_input(w)

@@ -1,6 +1,6 @@
 // tdq_quantize_act: token-group dual-constraint activation quantizer (Algorithm S1 steps 1-7).
 //
-// Three kernels:
+// Four kernels:
 //   * act_g32_ring_kernel   the fast path on dense rows (row stride == C): persistent, two CTAs per
 //     SM; one producer lane streams 16 KB tiles of 256 groups into a shared-memory ring with 1-D
 //     bulk copies and mbarrier transaction counts, eight consumer warps take one group per thread
@@ -12,6 +12,8 @@
 //     registers: max, sums, a pruned sorting network for the rank-k magnitude, the DCRP
 //     projection, an exact quotient, round-half-even, and one 128-bit store of 32 nibbles.
 //     One pass over HBM: 2 (bf16) or 4 (fp32) bytes in, 0.5 + 0.125 bytes out per element.
+//   * act_g32_nchw_kernel   channel-major input [B, C, H*W]: a tile of 32 channel rows is staged in
+//     shared memory and each thread gathers one position's 32 channels (tdq_quantize_act_nchw).
 //   * act_generic_kernel   any even g <= 4096, any C, any alignment: one warp per group,
 //     rank selection by bisection on the bit patterns of |x|, IEEE division.
 //
@@ -341,6 +343,83 @@ cudaError_t launch_fast(const ActArgs& a, cudaStream_t st) {
     return cudaGetLastError();
 }
 
+// ------------------------------------------------------------------------------------------
+// channel-major input: x is [B][C][H*W] (a convolutional feature map) and is quantized along C
+// without a permuted copy.  A CTA takes one group of 32 channels and 256 consecutive positions of
+// one image: the 32 channel rows are read with coalesced loads into a shared-memory tile, then
+// thread t gathers position t's 32 channels down the tile's columns and quantizes them like any
+// other group.  Codes and scales come out token-major, [B*H*W, C/2] and [B*H*W, C/32].
+
+struct NchwArgs {
+    ActArgs a;          // x, K, k_zr, seven_tau, flags, codes, scale, offset
+    int64_t HW;         // positions per image
+    int32_t vec_ok;     // channel rows can be read with 16-byte loads
+};
+
+template <bool BF16, int KZR>
+__global__ void __launch_bounds__(kFastThreads) act_g32_nchw_kernel(NchwArgs n) {
+    constexpr int esz = BF16 ? 2 : 4;
+    constexpr int kRowBytes = kFastThreads * esz + 16;        // 16 bytes of padding per channel row
+    constexpr int kVecPerRow = kFastThreads * esz / 16;       // 16-byte pieces of a channel row
+    __shared__ __align__(16) uint8_t tile[32 * kRowBytes];
+    const ActArgs& a = n.a;
+    const int t = threadIdx.x;
+    const int64_t s0 = (int64_t)blockIdx.x * kFastThreads;    // first position of the tile
+    const int k = blockIdx.y;                                  // channel group
+    const int64_t b = blockIdx.z;
+    const uint8_t* img = reinterpret_cast<const uint8_t*>(a.x) + ((b * a.C + (int64_t)k * 32) * n.HW + s0) * esz;
+    const int64_t left = n.HW - s0;                            // positions from s0 to the end of the image
+    if (n.vec_ok) {
+#pragma unroll
+        for (int j = 0; j < 32 * kVecPerRow / kFastThreads; ++j) {
+            const int idx = t + j * kFastThreads;
+            const int c = idx / kVecPerRow, piece = idx % kVecPerRow;
+            uint4 v = make_uint4(0u, 0u, 0u, 0u);
+            if ((int64_t)(piece + 1) * (16 / esz) <= left)     // HW is a multiple of 16 bytes here: pieces are whole
+                v = __ldg(reinterpret_cast<const uint4*>(img + (int64_t)c * n.HW * esz) + piece);
+            *reinterpret_cast<uint4*>(tile + c * kRowBytes + piece * 16) = v;
+        }
+    } else {
+#pragma unroll 4
+        for (int c = 0; c < 32; ++c) {
+            const uint8_t* src = img + ((int64_t)c * n.HW + t) * esz;
+            if (BF16)
+                *reinterpret_cast<uint16_t*>(tile + c * kRowBytes + t * 2) =
+                    t < left ? __ldg(reinterpret_cast<const uint16_t*>(src)) : (uint16_t)0;
+            else
+                *reinterpret_cast<uint32_t*>(tile + c * kRowBytes + t * 4) =
+                    t < left ? __ldg(reinterpret_cast<const uint32_t*>(src)) : 0u;
+        }
+    }
+    __syncthreads();
+    if (t >= left) return;
+    uint32_t w[BF16 ? 16 : 32];
+    if (BF16) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const uint32_t lo = *reinterpret_cast<const uint16_t*>(tile + (2 * i) * kRowBytes + t * 2);
+            const uint32_t hi = *reinterpret_cast<const uint16_t*>(tile + (2 * i + 1) * kRowBytes + t * 2);
+            w[i] = lo | (hi << 16);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) w[i] = *reinterpret_cast<const uint32_t*>(tile + i * kRowBytes + t * 4);
+    }
+    process_group<BF16, KZR>(w, a, ((b * n.HW + s0 + t) * a.K) + k);
+}
+
+template <bool BF16>
+cudaError_t launch_nchw(const NchwArgs& n, int64_t B, cudaStream_t st) {
+    dim3 grid((unsigned)((n.HW + kFastThreads - 1) / kFastThreads), (unsigned)n.a.K, (unsigned)B);
+    switch (n.a.k_zr) {
+#define TDQ_CASE(KZ) case KZ: act_g32_nchw_kernel<BF16, KZ><<<grid, kFastThreads, 0, st>>>(n); break;
+        TDQ_CASE(4) TDQ_CASE(7) TDQ_CASE(10) TDQ_CASE(13) TDQ_CASE(16) TDQ_CASE(32)
+#undef TDQ_CASE
+        default: return cudaErrorInvalidValue;
+    }
+    return cudaGetLastError();
+}
+
 bool fast_rank(int k) { return k == 4 || k == 7 || k == 10 || k == 13 || k == 16 || k == 32; }
 
 }  // namespace
@@ -426,6 +505,47 @@ extern "C" tdq_status tdq_quantize_act(const void* x, tdq_dtype x_dtype, int64_t
             act_generic_kernel<false><<<(unsigned)blocks, kGenericWarps * 32, smem, stream>>>(a);
         e = cudaGetLastError();
     }
+    if (e != cudaSuccess) return TDQ_ERR_CUDA;
+    g_launch_count.fetch_add(1, std::memory_order_relaxed);
+    return TDQ_OK;
+}
+
+extern "C" tdq_status tdq_quantize_act_nchw(const void* x, tdq_dtype x_dtype, int64_t B, int64_t C, int64_t H, int64_t W,
+                                            const tdq_act_params* p, uint8_t* codes, float* scale, float* offset,
+                                            void* cuda_stream) {
+    if (H < 0 || W < 0) return TDQ_ERR_INVALID_ARG;
+    const int64_t HW = H * W;
+    if (B >= 0 && C > 0 && p && B * HW == 0) return TDQ_OK;   // an empty map: nothing to read, x may be null
+    tdq_status st = check_act_args(x, x_dtype, B, HW, C, C, p);
+    if (st != TDQ_OK) return st;
+    if (!codes || !scale) return TDQ_ERR_INVALID_ARG;
+    if (B * HW == 0) return TDQ_OK;
+    const int32_t g = p->group_size;
+    // the channel-major kernel is the fast path only: 32-channel groups, max-abs base radius, a rank it has
+    if (g != 32 || C % 32 != 0 || rank_of(p->base_percentile, g) != g || reinterpret_cast<uintptr_t>(codes) % 16 ||
+        ((p->flags & TDQ_ENABLE_C2) && !fast_rank(rank_of(p->zr, g))))
+        return TDQ_ERR_UNSUPPORTED;
+    if (C / 32 > 65535 || B > 65535 || (HW + kFastThreads - 1) / kFastThreads > INT32_MAX) return TDQ_ERR_UNSUPPORTED;
+    NchwArgs n;
+    n.a.x = x;
+    n.a.M = B * HW;
+    n.a.C = C;
+    n.a.row_stride = C;
+    n.a.g = g;
+    n.a.K = (int32_t)(C / 32);
+    n.a.total_groups = n.a.M * n.a.K;
+    n.a.k_zr = (p->flags & TDQ_ENABLE_C2) ? rank_of(p->zr, g) : 7;   // rank unused without C2; pick an instantiated kernel
+    n.a.k_base = g;
+    n.a.seven_tau = 7.0f * p->tau;
+    n.a.flags = p->flags;
+    n.a.codes = codes;
+    n.a.scale = scale;
+    n.a.offset = offset;
+    n.HW = HW;
+    const int64_t esz = x_dtype == TDQ_BF16 ? 2 : 4;
+    n.vec_ok = (reinterpret_cast<uintptr_t>(x) % 16 == 0 && (HW * esz) % 16 == 0) ? 1 : 0;
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    const cudaError_t e = (x_dtype == TDQ_BF16) ? launch_nchw<true>(n, B, stream) : launch_nchw<false>(n, B, stream);
     if (e != cudaSuccess) return TDQ_ERR_CUDA;
     g_launch_count.fetch_add(1, std::memory_order_relaxed);
     return TDQ_OK;

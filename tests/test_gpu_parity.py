@@ -281,3 +281,56 @@ def test_fused_settings_and_refusals(tdq):
     with pytest.raises(tdq.TdqError) as e:
         tdq.quant_linear_fused(wide, wcw, wsw)
     assert e.value.code == tdq.ERR_UNSUPPORTED
+
+
+# ------------------------------------------------------------------------------------------
+# channel-major input (feature maps quantized along C in place)
+
+def _feature_map(seed, B, C, H, W, bf16):
+    rng = np.random.RandomState(seed)
+    sig = np.exp(rng.normal(0.0, 0.7, size=(B, 1, H, W)))
+    x = (rng.normal(size=(B, C, H, W)) * sig).astype(np.float32)
+    x[rng.rand(B, C, H, W) < 0.02] *= 30.0          # a few outliers
+    x[:, :, 0, 0] = 0.0                              # an all-zero token
+    return si.f32_to_bf16_bits(x) if bf16 else x
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("B,C,H,W,bf16", [
+    (2, 64, 9, 16, True),      # 288-byte channel rows: vector loads, one tile with a tail
+    (3, 32, 20, 20, True),     # 400 positions: two tiles, the second ragged
+    (1, 96, 7, 9, False),      # 252-byte rows: element-wise loads
+    (2, 64, 8, 8, False),      # fp32 vector loads
+    (1, 320, 5, 13, True),     # 130-byte rows: element-wise loads, ten groups
+])
+def test_quantizer_channel_major_matches_oracle_and_the_row_major_path(tdq, B, C, H, W, bf16):
+    x = _feature_map(B * 1000 + C + H, B, C, H, W, bf16)
+    ref = oracle.quantize_act_nchw(x)
+    xt = to_cuda(x, bf16=bf16)
+    codes, scale = tdq.quantize_act_nchw(xt)
+    rows = xt.permute(0, 2, 3, 1).contiguous().view(B * H * W, C)
+    codes2, scale2 = tdq.quantize_act(rows)
+    assert torch.equal(codes, codes2) and torch.equal(scale.view(torch.int32), scale2.view(torch.int32))
+    x_tok = np.ascontiguousarray(np.transpose(x, (0, 2, 3, 1))).reshape(B * H * W, C)
+    compare_quantizer(_f32(x_tok, bf16), 32, ref, codes.cpu().numpy(), scale.cpu().numpy())
+
+
+@pytest.mark.gpu
+def test_quantizer_channel_major_settings_and_refusals(tdq):
+    x = _feature_map(7, 2, 64, 6, 8, True)
+    xt = to_cuda(x, bf16=True)
+    for tau, zr, flags in [(0.25, 0.2, 3), (1.0, 0.5, 3), (1.0, 0.2, 1), (1.0, 0.2, 0)]:
+        p = tdq.act_params(tau=tau, zr=zr, flags=flags)
+        ref = oracle.quantize_act_nchw(x, tau=tau, zr=zr, flags=flags)
+        codes, scale = tdq.quantize_act_nchw(xt, p)
+        np.testing.assert_array_equal(codes.cpu().numpy(), ref["codes"])
+        np.testing.assert_array_equal(scale.cpu().numpy(), ref["scale"])
+    for bad in (tdq.act_params(g=64), tdq.act_params(p=0.9), tdq.act_params(zr=0.25)):   # rank 8 has no fast kernel
+        with pytest.raises(tdq.TdqError) as e:
+            tdq.quantize_act_nchw(xt, bad)
+        assert e.value.code == tdq.ERR_UNSUPPORTED
+    # offsets are written when asked for, and an empty map is a no-op
+    off = torch.full((2 * 48, 2), 5.0, device="cuda")
+    tdq.quantize_act_nchw(xt, offset=off)
+    assert float(off.abs().max()) == 0.0
+    tdq.quantize_act_nchw(torch.empty((0, 64, 6, 8), dtype=torch.bfloat16, device="cuda"))

@@ -317,3 +317,19 @@ def test_linear_equals_float64_product_of_dequantized_operands(C, O, g):
     # a transposed or mis-indexed weight would break this asymmetric check
     nb = oracle.w4a4_linear(xa["codes"], xa["scale"], wq["codes"], wq["scale"], g=g)
     np.testing.assert_allclose(nb["y_d"], want - bias, rtol=0, atol=float(1e-12 * scale_ref.max()))
+
+
+def test_channel_major_wrapper_is_the_per_token_definition():
+    """quantize_act_nchw must treat x[b, :, h, w] as one token (Supp. S1.1's 4-D branch), with token
+    index (b*H + h)*W + w: checked token by token with plain indexing, no transpose."""
+    rng = np.random.RandomState(5)
+    B, C, H, W = 2, 64, 3, 5
+    x = rng.normal(size=(B, C, H, W)).astype(np.float32)
+    out = oracle.quantize_act_nchw(x)
+    for b in range(B):
+        for h in range(H):
+            for w in range(W):
+                one = oracle.quantize_act(np.array([x[b, c, h, w] for c in range(C)], np.float32)[None, :])
+                t = (b * H + h) * W + w
+                np.testing.assert_array_equal(out["codes"][t], one["codes"][0])
+                np.testing.assert_array_equal(out["scale"][t], one["scale"][0])
