@@ -439,6 +439,9 @@ def run_tdq(args):
             pf = tdq.act_params(flags=flags)
             q_switch_ms[label] = time_graph(lambda i: tdq.quantize_act(xi[i % n_iso], pf, codes=codes[i % nsets],
                                                                        scale=scales[i % nsets]), 4 * n_iso)
+        # the fixed-radius control: no reductions, the speed limit of a one-pass quantizer of this size
+        q_switch_ms["fixed_radius"] = time_graph(lambda i: tdq.quantize_act_fixed(xi[i % n_iso], 1.0, 32, codes=codes[i % nsets],
+                                                                                 scale=scales[i % nsets]), 4 * n_iso)
         del xi
         # channel-major input of the same volume: a [B, C, 24, 24] feature map quantized along C in place
         fm = [torch.randn((32, C, 24, 24), device=dev).mul_(torch.randn((32, 1, 24, 24), device=dev).exp_())

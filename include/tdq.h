@@ -99,6 +99,22 @@ tdq_status tdq_quantize_act_nchw(const void* x, tdq_dtype x_dtype, int64_t B, in
                                  float* scale, float* offset, void* cuda_stream);
 
 /*
+ * Fixed-radius control (the fixed offline-calibrated variant of Supp. S1.2 and S4.2): the clip
+ * radius is a number chosen beforehand for the whole layer, so nothing is reduced over the
+ * activations.  With c = max(radius, 1e-8) in every group:
+ *   Delta = max(c/7, 1e-8);  q = clip(round_half_even(clip(x,-c,c) / Delta), -8, 7).
+ *   x, B, N, C, row_stride_elems as for tdq_quantize_act;  codes [B*N, C/2];  scale [B*N, C/g]
+ *   (every entry Delta, so that the outputs feed tdq_w4a4_linear unchanged);  offset NULL or
+ *   [B*N, C/g], filled with 0.
+ * TDQ_ERR_INVALID_ARG for null pointers, radius <= 0 or a bad group size; TDQ_ERR_UNSUPPORTED
+ * unless group_size % 8 == 0, C % group_size == 0, x is 16-byte aligned with a row pitch that is
+ * a multiple of 16 bytes, and codes is 4-byte aligned.
+ */
+tdq_status tdq_quantize_act_fixed(const void* x, tdq_dtype x_dtype, int64_t B, int64_t N, int64_t C,
+                                  int64_t row_stride_elems, int32_t group_size, float radius,
+                                  uint8_t* codes, float* scale, float* offset, void* cuda_stream);
+
+/*
  * Static weight quantizer, Eq. 4 with absmax per-output-channel scales:
  *   s_o = max(max_i |W[o,i]| / 7, 1e-8);  Q = clip(round_half_even(W / s_o), -8, 7).
  *   w       [O, I] row-major, contiguous, w_dtype.

@@ -49,6 +49,8 @@ def _load():
             lib.tdq_oracle_quantize_act.argtypes = [vp, ctypes.c_int, i64, i64, i64, i32, f32, f32,
                                                     f32, u32, vp, vp, vp, vp, vp]
             lib.tdq_oracle_quantize_act.restype = ctypes.c_int
+            lib.tdq_oracle_quantize_act_fixed.argtypes = [vp, ctypes.c_int, i64, i64, i64, i32, f32, vp, vp, vp]
+            lib.tdq_oracle_quantize_act_fixed.restype = ctypes.c_int
             lib.tdq_oracle_quantize_weight.argtypes = [vp, ctypes.c_int, i64, i64, i32, vp, vp, vp]
             lib.tdq_oracle_quantize_weight.restype = ctypes.c_int
             lib.tdq_oracle_w4a4_linear.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, i32, vp, vp, vp, vp]
@@ -103,6 +105,24 @@ def quantize_act(x, g=32, tau=1.0, zr=0.2, p=1.0, flags=ENABLE_C1 | ENABLE_C2, C
                                          _ptr(out["scale"]), _ptr(out["clip"]), _ptr(out["active"]))
     if rc != 0:
         raise ValueError("tdq_oracle_quantize_act rejected its arguments")
+    return out
+
+
+def quantize_act_fixed(x, radius, g=32, C=None):
+    """The fixed-radius control: steps 5-9 of Algorithm S1 with the same given clip radius in every group.
+    Returns a dict: q int8 [M, C_pad], codes uint8 [M, C_pad/2], scale float32 [M, K]."""
+    x, dt = _as_input(x)
+    row_stride = x.shape[-1]
+    C = row_stride if C is None else int(C)
+    M = int(np.prod(x.shape[:-1])) if x.ndim > 1 else 1
+    K = (C + g - 1) // g
+    C_pad = K * g
+    out = dict(q=np.empty((M, C_pad), np.int8), codes=np.empty((M, C_pad // 2), np.uint8),
+               scale=np.empty((M, K), np.float32))
+    rc = _load().tdq_oracle_quantize_act_fixed(_ptr(x), dt, M, C, row_stride, g, float(radius),
+                                               _ptr(out["q"]), _ptr(out["codes"]), _ptr(out["scale"]))
+    if rc != 0:
+        raise ValueError("tdq_oracle_quantize_act_fixed rejected its arguments")
     return out
 
 

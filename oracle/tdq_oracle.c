@@ -15,6 +15,8 @@
  *                               floor, 1e-8 clip floor, population std + 1e-12,
  *                               round-half-to-even) and the rank rule of
  *                               Supp. S2.2 (k = ceil(p*g), 1-indexed).
+ *   tdq_oracle_quantize_act_fixed  the same steps 5-9 with a radius fixed beforehand
+ *                               (the fixed offline-calibrated control of Supp. S1.2).
  *   tdq_oracle_quantize_weight  Eq. 4 with absmax per-output-channel scales.
  *   tdq_oracle_w4a4_linear      Algorithm S1 step 10 with x_hat = Delta_k * q
  *                               (Eq. 9) and W_hat = s_o * Q_w (Eq. 4) substituted,
@@ -184,6 +186,46 @@ int tdq_oracle_quantize_act(const void* x, int x_dtype, int64_t M, int64_t C,
         free(xg); free(ag); free(qg);
     }
     return status;
+}
+
+/*
+ * Fixed-radius control (Supp. S1.2, "fixed controls"; Supp. S4.2's fixed offline calibration row):
+ * the clip radius is a number fixed beforehand for the whole layer instead of being computed from
+ * the activations.  Steps 5-9 of Algorithm S1 with c = max(radius, 1e-8) in every group:
+ *   Delta = max(c / 7, 1e-8);  q = clip(rint(clip(x, -c, c) / Delta), -8, 7).
+ * Outputs as for tdq_oracle_quantize_act (scale holds the same Delta in every entry).
+ */
+int tdq_oracle_quantize_act_fixed(const void* x, int x_dtype, int64_t M, int64_t C,
+                                  int64_t row_stride, int32_t g, float radius, int8_t* q,
+                                  uint8_t* codes, float* scale) {
+    if (!x || M < 0 || C <= 0 || g <= 0 || (g & 1) || row_stride < C || !(radius > 0.0f)) return -1;
+    const int64_t K = (C + g - 1) / g;
+    const int64_t C_pad = K * g;
+    float c = radius;
+    if (c < 1e-8f) c = 1e-8f;
+    float delta = c / 7.0f;
+    if (delta < 1e-8f) delta = 1e-8f;
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m) {
+        for (int64_t ch = 0; ch < C_pad; ch += 2) {
+            int qi[2];
+            for (int j = 0; j < 2; ++j) {
+                float xt = (ch + j < C) ? load_elem(x, x_dtype, m * row_stride + ch + j) : 0.0f;
+                if (xt > c) xt = c;
+                if (xt < -c) xt = -c;
+                float rr = rintf(xt / delta);
+                int v = (int)rr;
+                if (v > Q_MAX) v = Q_MAX;
+                if (v < Q_MIN) v = Q_MIN;
+                qi[j] = v;
+                if (q) q[m * C_pad + ch + j] = (int8_t)v;
+            }
+            if (codes) codes[(m * C_pad + ch) / 2] = (uint8_t)(nibble(qi[0]) | (nibble(qi[1]) << 4));
+        }
+        if (scale)
+            for (int64_t k = 0; k < K; ++k) scale[m * K + k] = delta;
+    }
+    return 0;
 }
 
 /*

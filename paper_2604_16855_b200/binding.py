@@ -22,7 +22,7 @@ ENABLE_C1, ENABLE_C2 = 1, 2
 
 # every symbol include/tdq.h declares
 EXPORTS = ["tdq_default_act_params", "tdq_quantize_act", "tdq_quantize_weight", "tdq_w4a4_linear",
-           "tdq_quant_linear_fused", "tdq_quant_linear_host", "tdq_quantize_act_nchw", "tdq_linear_workspace_bytes",
+           "tdq_quant_linear_fused", "tdq_quant_linear_host", "tdq_quantize_act_nchw", "tdq_quantize_act_fixed", "tdq_linear_workspace_bytes",
            "tdq_workspace_status", "tdq_status_string", "tdq_kernel_launch_count", "tdq_w4a4_linear_static"]
 
 
@@ -39,6 +39,8 @@ _lib.tdq_quantize_act.argtypes = [_vp, ctypes.c_int, _i64, _i64, _i64, _i64, _pp
 _lib.tdq_quantize_act.restype = ctypes.c_int
 _lib.tdq_quantize_act_nchw.argtypes = [_vp, ctypes.c_int, _i64, _i64, _i64, _i64, _pp, _vp, _vp, _vp, _vp]
 _lib.tdq_quantize_act_nchw.restype = ctypes.c_int
+_lib.tdq_quantize_act_fixed.argtypes = [_vp, ctypes.c_int, _i64, _i64, _i64, _i64, _i32, ctypes.c_float, _vp, _vp, _vp, _vp]
+_lib.tdq_quantize_act_fixed.restype = ctypes.c_int
 _lib.tdq_quantize_weight.argtypes = [_vp, ctypes.c_int, _i64, _i64, _i32, _vp, _vp, _vp]
 _lib.tdq_quantize_weight.restype = ctypes.c_int
 _lib.tdq_w4a4_linear.argtypes = [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp, ctypes.c_int, _i64,
@@ -141,6 +143,22 @@ def quantize_act(x: torch.Tensor, params: ActParams | None = None, *, codes=None
     stride = x2.stride(0) if M > 1 else C
     _check(_lib.tdq_quantize_act(_ptr(x2), _dtype_id(x2), 1, M, C, stride, ctypes.byref(p), _ptr(codes),
                                  _ptr(scale), _ptr(offset), _stream(x)), "tdq_quantize_act")
+    return codes, scale
+
+
+def quantize_act_fixed(x: torch.Tensor, radius: float, g: int = 32, *, codes=None, scale=None, offset=None):
+    """tdq_quantize_act_fixed: the same clip radius in every group.  Returns (codes [M, C/2], scale [M, C/g])."""
+    _need_cuda(x, codes, scale, offset)
+    C = x.shape[-1]
+    x2 = x.reshape(-1, C)
+    M = x2.shape[0]
+    if codes is None:
+        codes = torch.empty((M, C // 2), dtype=torch.uint8, device=x.device)
+    if scale is None:
+        scale = torch.empty((M, max(C // g, 1)), dtype=torch.float32, device=x.device)
+    stride = x2.stride(0) if M > 1 else C
+    _check(_lib.tdq_quantize_act_fixed(_ptr(x2), _dtype_id(x2), 1, M, C, stride, g, radius, _ptr(codes), _ptr(scale),
+                                       _ptr(offset), _stream(x)), "tdq_quantize_act_fixed")
     return codes, scale
 
 

@@ -1,6 +1,6 @@
 // tdq_quantize_act: token-group dual-constraint activation quantizer (Algorithm S1 steps 1-7).
 //
-// Four kernels:
+// Five kernels:
 //   * act_g32_ring_kernel   the fast path on dense rows (row stride == C): persistent, two CTAs per
 //     SM; one producer lane streams 16 KB tiles of 256 groups into a shared-memory ring with 1-D
 //     bulk copies and mbarrier transaction counts, eight consumer warps take one group per thread
@@ -14,6 +14,8 @@
 //     One pass over HBM: 2 (bf16) or 4 (fp32) bytes in, 0.5 + 0.125 bytes out per element.
 //   * act_g32_nchw_kernel   channel-major input [B, C, H*W]: a tile of 32 channel rows is staged in
 //     shared memory and each thread gathers one position's 32 channels (tdq_quantize_act_nchw).
+//   * act_fixed_kernel   the fixed-radius control: no reductions, 8 channels per thread
+//     (tdq_quantize_act_fixed).
 //   * act_generic_kernel   any even g <= 4096, any C, any alignment: one warp per group,
 //     rank selection by bisection on the bit patterns of |x|, IEEE division.
 //
@@ -420,6 +422,72 @@ cudaError_t launch_nchw(const NchwArgs& n, int64_t B, cudaStream_t st) {
     return cudaGetLastError();
 }
 
+// ------------------------------------------------------------------------------------------
+// fixed-radius control: no reductions at all.  A thread takes 8 consecutive channels of a row:
+// one or two 16-byte loads, eight exact quotients, one 4-byte store of codes.
+
+struct FixedArgs {
+    const void* x;
+    int64_t M, C, row_stride;   // elements
+    int64_t chunks_per_row;     // C / 8
+    int32_t g, K;
+    float c, delta;
+    uint8_t* codes;
+    float* scale;
+    float* offset;
+};
+
+template <bool BF16>
+__global__ void __launch_bounds__(256) act_fixed_kernel(FixedArgs f) {
+    const int64_t idx = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (idx >= f.M * f.chunks_per_row) return;
+    int64_t m, ch8;
+    if (f.M * f.chunks_per_row <= 0xffffffffll) {   // the usual case: 32-bit division
+        const uint32_t q32 = (uint32_t)idx / (uint32_t)f.chunks_per_row;
+        m = q32;
+        ch8 = (uint32_t)idx - q32 * (uint32_t)f.chunks_per_row;
+    } else {
+        m = idx / f.chunks_per_row;
+        ch8 = idx - m * f.chunks_per_row;
+    }
+    float v[8];
+    if (BF16) {
+        const uint4 t = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const uint16_t*>(f.x) + m * f.row_stride + ch8 * 8));
+        const uint32_t w[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            v[2 * i] = __uint_as_float(w[i] << 16);
+            v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+        }
+    } else {
+        const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const float*>(f.x) + m * f.row_stride + ch8 * 8);
+        const uint4 t0 = __ldg(src), t1 = __ldg(src + 1);
+        v[0] = __uint_as_float(t0.x); v[1] = __uint_as_float(t0.y); v[2] = __uint_as_float(t0.z); v[3] = __uint_as_float(t0.w);
+        v[4] = __uint_as_float(t1.x); v[5] = __uint_as_float(t1.y); v[6] = __uint_as_float(t1.z); v[7] = __uint_as_float(t1.w);
+    }
+    uint32_t word = 0u;
+    if (f.delta <= 1e30f) {   // two channels at a time, as in the token-group kernels
+        const float rcp = __frcp_rn(f.delta);
+        const uint64_t rcp2 = f2_pack(rcp, rcp), neg_delta2 = f2_pack(-f.delta, -f.delta);
+        const uint64_t magic2 = f2_pack(kRoundMagic8, kRoundMagic8);
+        uint32_t acc = 0u;
+#pragma unroll
+        for (int n = 6; n >= 0; n -= 2)
+            nibbles_fast2(f2_pack(fminf(fmaxf(v[n], -f.c), f.c), fminf(fmaxf(v[n + 1], -f.c), f.c)), neg_delta2, rcp2, magic2, acc);
+        word = pack_word(acc);
+    } else {                  // 1 / Delta would be subnormal: take the IEEE division
+#pragma unroll
+        for (int n = 0; n < 8; ++n) word |= nibble_ieee(v[n], f.c, f.delta) << (4 * n);
+    }
+    reinterpret_cast<uint32_t*>(f.codes)[idx] = word;
+    const int64_t ch = ch8 * 8;
+    if (ch % f.g == 0) {
+        const int64_t gi = m * f.K + ch / f.g;
+        f.scale[gi] = f.delta;
+        if (f.offset) f.offset[gi] = 0.0f;
+    }
+}
+
 bool fast_rank(int k) { return k == 4 || k == 7 || k == 10 || k == 13 || k == 16 || k == 32; }
 
 }  // namespace
@@ -547,6 +615,37 @@ extern "C" tdq_status tdq_quantize_act_nchw(const void* x, tdq_dtype x_dtype, in
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
     const cudaError_t e = (x_dtype == TDQ_BF16) ? launch_nchw<true>(n, B, stream) : launch_nchw<false>(n, B, stream);
     if (e != cudaSuccess) return TDQ_ERR_CUDA;
+    g_launch_count.fetch_add(1, std::memory_order_relaxed);
+    return TDQ_OK;
+}
+
+extern "C" tdq_status tdq_quantize_act_fixed(const void* x, tdq_dtype x_dtype, int64_t B, int64_t N, int64_t C,
+                                             int64_t row_stride_elems, int32_t group_size, float radius, uint8_t* codes,
+                                             float* scale, float* offset, void* cuda_stream) {
+    if (!x || !codes || !scale) return TDQ_ERR_INVALID_ARG;
+    if (x_dtype != TDQ_F32 && x_dtype != TDQ_BF16) return TDQ_ERR_INVALID_ARG;
+    if (B < 0 || N < 0 || C <= 0 || row_stride_elems < C) return TDQ_ERR_INVALID_ARG;
+    if (group_size < 2 || group_size > 4096 || (group_size & 1) || !(radius > 0.0f)) return TDQ_ERR_INVALID_ARG;
+    const int64_t M = B * N;
+    if (M == 0) return TDQ_OK;
+    const int64_t esz = x_dtype == TDQ_BF16 ? 2 : 4;
+    if (group_size % 8 || C % group_size || reinterpret_cast<uintptr_t>(x) % 16 || (row_stride_elems * esz) % 16 ||
+        reinterpret_cast<uintptr_t>(codes) % 4)
+        return TDQ_ERR_UNSUPPORTED;
+    FixedArgs f;
+    f.x = x; f.M = M; f.C = C; f.row_stride = row_stride_elems; f.chunks_per_row = C / 8;
+    f.g = group_size; f.K = (int32_t)(C / group_size);
+    f.c = fmaxf(radius, kClipFloor);
+    f.delta = fmaxf(f.c / kQmax, kStepFloor);      // binary32 division on the host: the same IEEE operation
+    f.codes = codes; f.scale = scale; f.offset = offset;
+    const int64_t blocks = (M * f.chunks_per_row + 255) / 256;
+    if (blocks > INT32_MAX) return TDQ_ERR_UNSUPPORTED;
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    if (x_dtype == TDQ_BF16)
+        act_fixed_kernel<true><<<(unsigned)blocks, 256, 0, stream>>>(f);
+    else
+        act_fixed_kernel<false><<<(unsigned)blocks, 256, 0, stream>>>(f);
+    if (cudaGetLastError() != cudaSuccess) return TDQ_ERR_CUDA;
     g_launch_count.fetch_add(1, std::memory_order_relaxed);
     return TDQ_OK;
 }

@@ -334,3 +334,41 @@ def test_quantizer_channel_major_settings_and_refusals(tdq):
     tdq.quantize_act_nchw(xt, offset=off)
     assert float(off.abs().max()) == 0.0
     tdq.quantize_act_nchw(torch.empty((0, 64, 6, 8), dtype=torch.bfloat16, device="cuda"))
+
+
+# ------------------------------------------------------------------------------------------
+# fixed-radius control
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("idx,bf16,g,radius", [(1, False, 32, 1.0), (2, True, 32, 0.37), (3, True, 64, 3.0),
+                                               (3, True, 320, 0.05), (2, True, 8, 1e-9), (1, False, 32, 1e38)])
+def test_fixed_radius_quantizer_matches_oracle(tdq, idx, bf16, g, radius):
+    case = si.config(idx)
+    x = case.x.reshape(-1, case.C)[:3000]
+    ref = oracle.quantize_act_fixed(x, radius, g=g)
+    codes, scale = tdq.quantize_act_fixed(to_cuda(x, bf16=bf16), radius, g)
+    np.testing.assert_array_equal(codes.cpu().numpy(), ref["codes"])
+    np.testing.assert_array_equal(scale.cpu().numpy(), ref["scale"])
+
+
+@pytest.mark.gpu
+def test_fixed_radius_quantizer_stride_offset_linear_and_refusals(tdq):
+    case = si.config3()
+    x = case.x.reshape(-1, case.C)[:520]
+    wide = np.zeros((520, case.C + 24), np.uint16)
+    wide[:, :case.C] = x
+    xt = to_cuda(wide, bf16=True)[:, :case.C]                 # rows 344 elements apart
+    off = torch.full((520, case.C // 32), 3.0, device="cuda")
+    codes, scale = tdq.quantize_act_fixed(xt, 2.0, 32, offset=off)
+    ref = oracle.quantize_act_fixed(x, 2.0, g=32)
+    np.testing.assert_array_equal(codes.cpu().numpy(), ref["codes"])
+    assert float(off.abs().max()) == 0.0
+    # the outputs feed the linear layer unchanged
+    wc, ws = tdq.quantize_weight(to_cuda(case.w))
+    y = tdq.w4a4_linear(codes, scale, wc, ws)
+    wq = oracle.quantize_weight(case.w)
+    compare_y(y.cpu().numpy(), oracle.w4a4_linear(ref["codes"], ref["scale"], wq["codes"], wq["scale"]), case.C // 32)
+    for g, radius, code in [(12, 1.0, tdq.ERR_UNSUPPORTED), (32, 0.0, tdq.ERR_INVALID_ARG), (96, 1.0, tdq.ERR_UNSUPPORTED)]:
+        with pytest.raises(tdq.TdqError) as e:
+            tdq.quantize_act_fixed(xt, radius, g)
+        assert e.value.code == code

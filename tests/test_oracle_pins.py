@@ -333,3 +333,26 @@ def test_channel_major_wrapper_is_the_per_token_definition():
                 t = (b * H + h) * W + w
                 np.testing.assert_array_equal(out["codes"][t], one["codes"][0])
                 np.testing.assert_array_equal(out["scale"][t], one["scale"][0])
+
+
+def test_fixed_radius_control_against_the_token_group_path_and_its_bounds():
+    """Pins for quantize_act_fixed.  (a) When every group's largest magnitude equals the fixed radius, the
+    token-group quantizer without DCRP (flags = 0) chooses exactly that radius itself, so both must give the
+    same codes and steps.  (b) Inside the radius the reconstruction error is at most half a step, outside
+    the codes saturate at +-7, zeros stay zero."""
+    rng = np.random.RandomState(3)
+    M, C, g, radius = 40, 96, 32, 2.5
+    x = rng.uniform(-radius, radius, size=(M, C)).astype(np.float32)
+    x[:, ::g] = np.where(rng.rand(M, C // g) < 0.5, radius, -radius).astype(np.float32)   # plant the maximum in each group
+    fixed = oracle.quantize_act_fixed(x, radius, g=g)
+    dstg = oracle.quantize_act(x, g=g, flags=0)
+    np.testing.assert_array_equal(fixed["codes"], dstg["codes"])
+    np.testing.assert_array_equal(fixed["scale"], dstg["scale"])
+    delta = np.float32(radius) / np.float32(7.0)
+    assert np.all(fixed["scale"] == delta)
+    assert np.abs(fixed["q"].astype(np.float64) * float(delta) - x).max() <= float(delta) / 2 * (1 + 1e-6)
+    y = np.array([[0.0, 10.0, -10.0, radius * 1.0001] + [0.0] * 28], np.float32)
+    out = oracle.quantize_act_fixed(y, radius, g=g)
+    assert list(out["q"][0, :4]) == [0, 7, -7, 7]
+    with pytest.raises(ValueError):
+        oracle.quantize_act_fixed(y, 0.0)
