@@ -47,13 +47,18 @@ typedef enum { TDQ_F32 = 0, TDQ_BF16 = 1 } tdq_dtype;
  * variants of Table S6).  Both = COD-TDQ, neither = DSTG only. */
 #define TDQ_ENABLE_C1 1u  /* step-to-dispersion bound, Eq. 10 */
 #define TDQ_ENABLE_C2 2u  /* zero-bin mass bound, Eq. 11      */
+/* A variant, not the paper's quantizer: after the projection the step is rounded DOWN to a power of
+ * two, Delta' = 2^floor(log2 Delta), and c' = 7 Delta'.  Both DCRP bounds are upper bounds on c, so they
+ * still hold; the clip range shrinks by up to a factor of two.  Such steps let tdq_w4a4_linear_pow2
+ * fold the group scale into the tensor-core operand. */
+#define TDQ_POW2_STEP 4u
 
 typedef struct {
     int32_t group_size;      /* g, even, 2..4096; default 32.  g == C_pad gives one scale per token */
     float tau;               /* C1: Delta_k / sigma_k <= tau, tau > 0; default 1.0                   */
     float zr;                /* C2: zero-bin mass bound in (0,1]; default 0.2; rank ceil(zr*g)       */
     float base_percentile;   /* p in (0,1]; 1.0 = max-abs base radius, else rank ceil(p*g) (Eq. 6)   */
-    uint32_t flags;          /* TDQ_ENABLE_C1 | TDQ_ENABLE_C2                                        */
+    uint32_t flags;          /* TDQ_ENABLE_C1 | TDQ_ENABLE_C2 [| TDQ_POW2_STEP]                      */
 } tdq_act_params;
 
 /* The paper's shared setting (g, tau, zr) = (32, 1.0, 0.2), max-abs base radius, both bounds. */

@@ -24,6 +24,7 @@ F32 = 0
 BF16 = 1
 ENABLE_C1 = 1
 ENABLE_C2 = 2
+POW2_STEP = 4
 
 
 def build(force: bool = False) -> str:

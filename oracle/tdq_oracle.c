@@ -55,6 +55,7 @@
 #define ORACLE_BF16 1
 #define ORACLE_ENABLE_C1 1u
 #define ORACLE_ENABLE_C2 2u
+#define ORACLE_POW2_STEP 4u   /* variant: step rounded down to a power of two after the projection */
 
 #define Q_MAX 7
 #define Q_MIN (-8)
@@ -159,6 +160,13 @@ int tdq_oracle_quantize_act(const void* x, int x_dtype, int64_t M, int64_t C,
             /* Eq. 8 / Alg. S1 step 6. */
             float delta = c / 7.0f;
             if (delta < 1e-8f) delta = 1e-8f;
+            if (flags & ORACLE_POW2_STEP) {
+                /* not in the paper: Delta' = 2^floor(log2 Delta), c' = 7 Delta' <= c */
+                int e;
+                (void)frexpf(delta, &e);          /* delta = m * 2^e, m in [0.5, 1) */
+                delta = ldexpf(0.5f, e);
+                c = 7.0f * delta;
+            }
 
             /* steps 5 and 7. */
             for (int32_t i = 0; i < g; ++i) {

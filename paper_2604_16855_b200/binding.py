@@ -18,7 +18,7 @@ _lib = ctypes.CDLL(LIB_PATH)
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_DEVICE_TIMEOUT = range(7)
 F32, BF16 = 0, 1
-ENABLE_C1, ENABLE_C2 = 1, 2
+ENABLE_C1, ENABLE_C2, POW2_STEP = 1, 2, 4
 
 # every symbol include/tdq.h declares
 EXPORTS = ["tdq_default_act_params", "tdq_quantize_act", "tdq_quantize_weight", "tdq_w4a4_linear",

@@ -67,6 +67,10 @@ __device__ __forceinline__ void dcrp_project(float c_base, float sigma, float th
     cc = fmaxf(cc, kClipFloor);
     c = cc;
     delta = fmaxf(__fdiv_rn(cc, kQmax), kStepFloor);
+    if (flags & TDQ_POW2_STEP) {   // the power-of-two variant: drop the step's mantissa, keep c = 7 Delta
+        delta = __uint_as_float(__float_as_uint(delta) & 0xff800000u);
+        c = __fmul_rn(kQmax, delta);
+    }
 }
 
 // One element of Alg. S1 steps 5 and 7 with a true IEEE division; returns the code.

@@ -501,7 +501,7 @@ tdq_status check_act_args(const void* x, tdq_dtype dt, int64_t B, int64_t N, int
     if (p->group_size < 2 || p->group_size > 4096 || (p->group_size & 1)) return TDQ_ERR_INVALID_ARG;
     if (!(p->tau > 0.0f) || !(p->zr > 0.0f && p->zr <= 1.0f)) return TDQ_ERR_INVALID_ARG;
     if (!(p->base_percentile > 0.0f && p->base_percentile <= 1.0f)) return TDQ_ERR_INVALID_ARG;
-    if (p->flags & ~(TDQ_ENABLE_C1 | TDQ_ENABLE_C2)) return TDQ_ERR_INVALID_ARG;
+    if (p->flags & ~(TDQ_ENABLE_C1 | TDQ_ENABLE_C2 | TDQ_POW2_STEP)) return TDQ_ERR_INVALID_ARG;
     return TDQ_OK;
 }
 

@@ -372,3 +372,18 @@ def test_fixed_radius_quantizer_stride_offset_linear_and_refusals(tdq):
         with pytest.raises(tdq.TdqError) as e:
             tdq.quantize_act_fixed(xt, radius, g)
         assert e.value.code == code
+
+
+# ------------------------------------------------------------------------------------------
+# power-of-two step variant
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("idx,bf16,g", [(1, False, 32), (2, True, 32), (3, True, 32), (3, True, 64), (2, True, 16)])
+def test_power_of_two_steps_match_oracle(tdq, idx, bf16, g):
+    case = si.config(idx)
+    x = case.x.reshape(-1, case.C)[:2500]
+    flags = 7
+    ref, codes, scale = _quant_both(tdq, x, bf16, g=g, flags=flags)
+    np.testing.assert_array_equal(codes, ref["codes"])
+    np.testing.assert_array_equal(scale, ref["scale"])
+    assert np.all(np.frexp(scale.astype(np.float64))[0] == 0.5)

@@ -356,3 +356,24 @@ def test_fixed_radius_control_against_the_token_group_path_and_its_bounds():
     assert list(out["q"][0, :4]) == [0, 7, -7, 7]
     with pytest.raises(ValueError):
         oracle.quantize_act_fixed(y, 0.0)
+
+
+def test_power_of_two_step_variant_keeps_the_bounds_and_only_shrinks_the_range():
+    """Pins for the POW2_STEP variant: every step is a power of two with Delta/2 < Delta' <= Delta of the
+    paper's quantizer, c' = 7 Delta' <= c (so both DCRP bounds, which are upper bounds on c, still hold), and
+    the codes are what that grid gives: rint(clip(x, +-c') / Delta'), a division that is exact."""
+    case = si.config2()
+    x = case.x_f32().reshape(-1, case.C)[:800]
+    base = oracle.quantize_act(x)
+    pow2 = oracle.quantize_act(x, flags=oracle.ENABLE_C1 | oracle.ENABLE_C2 | oracle.POW2_STEP)
+    d, dp = base["scale"].astype(np.float64), pow2["scale"].astype(np.float64)
+    mant, _ = np.frexp(dp)
+    assert np.all(mant == 0.5)                                  # powers of two
+    assert np.all(dp <= d) and np.all(dp > d / 2)
+    assert np.all(pow2["clip"].astype(np.float64) == 7.0 * dp)
+    assert np.all(pow2["clip"] <= base["clip"])
+    K = case.C // 32
+    xg = x.astype(np.float64).reshape(-1, K, 32)
+    c = pow2["clip"].astype(np.float64)[:, :, None]
+    want = np.clip(np.rint(np.clip(xg, -c, c) / dp[:, :, None]), -8, 7).reshape(x.shape[0], -1)
+    np.testing.assert_array_equal(pow2["q"], want.astype(np.int8))
