@@ -153,6 +153,27 @@ tdq_status tdq_w4a4_linear(const uint8_t* xcodes, const float* xscale, const uin
                            void* cuda_stream);
 
 /*
+ * The linear layer for activations quantized with TDQ_POW2_STEP (a variant; the paper has no
+ * counterpart).  When every step of a token is a power of two, Delta[m,k] = 2^(e_m + s[m,k]), the
+ * group scale can ride inside the tensor-core operand: a code is stored as the FP8 (E4M3) value
+ * q * 2^(s - 9), which is exact for s in 0..14, the whole contraction accumulates in one fp32
+ * accumulator, and each row is scaled once, by 2^e_m * s_o, at the end.  There is no per-group pass
+ * over the accumulators, which is what bounds tdq_w4a4_linear at g = 32.
+ *   Arguments as for tdq_w4a4_linear (no acc_debug).  xscale entries must be positive powers of
+ *   two; anything else is reported through tdq_workspace_status (detail code 11) and the output
+ *   is then meaningless.
+ *   e_m is the largest step exponent of the row minus 14.  Steps more than 2^14 below the row's
+ *   largest lose low bits of their codes (truncation; the lost part is below 2^-14 of the row's
+ *   largest step per element).  Sums are accumulated in binary32 by the tensor core, in its
+ *   order: results agree with tdq_w4a4_linear on the same inputs to about 1e-6 relative to the sum
+ *   of the absolute terms, not bit for bit.
+ */
+tdq_status tdq_w4a4_linear_pow2(const uint8_t* xcodes, const float* xscale, const uint8_t* wcodes,
+                                const float* wscale, const float* bias, int64_t M, int64_t I_pad, int64_t O,
+                                int32_t group_size, void* y, tdq_dtype y_dtype, int64_t y_row_stride,
+                                void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Quantizer fused into the linear layer as the producer of its A operand (Algorithm S1 steps
  * 1-10 in one kernel, with no pass over the activations besides the layer's own): the same
  * result, bit for bit, as tdq_quantize_act followed by tdq_w4a4_linear, but activation codes

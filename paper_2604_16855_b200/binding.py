@@ -22,7 +22,7 @@ ENABLE_C1, ENABLE_C2, POW2_STEP = 1, 2, 4
 
 # every symbol include/tdq.h declares
 EXPORTS = ["tdq_default_act_params", "tdq_quantize_act", "tdq_quantize_weight", "tdq_w4a4_linear",
-           "tdq_quant_linear_fused", "tdq_quant_linear_host", "tdq_quantize_act_nchw", "tdq_quantize_act_fixed", "tdq_linear_workspace_bytes",
+           "tdq_quant_linear_fused", "tdq_quant_linear_host", "tdq_quantize_act_nchw", "tdq_quantize_act_fixed", "tdq_w4a4_linear_pow2", "tdq_linear_workspace_bytes",
            "tdq_workspace_status", "tdq_status_string", "tdq_kernel_launch_count", "tdq_w4a4_linear_static"]
 
 
@@ -46,6 +46,8 @@ _lib.tdq_quantize_weight.restype = ctypes.c_int
 _lib.tdq_w4a4_linear.argtypes = [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp, ctypes.c_int, _i64,
                                  _vp, _vp, _sz, _vp]
 _lib.tdq_w4a4_linear.restype = ctypes.c_int
+_lib.tdq_w4a4_linear_pow2.argtypes = [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp, ctypes.c_int, _i64, _vp, _sz, _vp]
+_lib.tdq_w4a4_linear_pow2.restype = ctypes.c_int
 _lib.tdq_w4a4_linear_static.argtypes = [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i32, _vp, ctypes.c_int, _i64,
                                         _i32, _vp]
 _lib.tdq_w4a4_linear_static.restype = ctypes.c_int
@@ -213,6 +215,22 @@ def w4a4_linear(xcodes, xscale, wcodes, wscale, bias=None, *, g=32, out_dtype=to
     _check(_lib.tdq_w4a4_linear(_ptr(xcodes), _ptr(xscale), _ptr(wcodes), _ptr(wscale), _ptr(bias), M, I_pad, O, g,
                                 _ptr(y), _dtype_id(y), y.stride(0) if M > 0 else O, _ptr(acc_debug),
                                 _ptr(workspace), workspace.numel(), _stream(xcodes)), "tdq_w4a4_linear")
+    return y
+
+
+def w4a4_linear_pow2(xcodes, xscale, wcodes, wscale, bias=None, *, g=32, out_dtype=torch.float32, y=None, workspace=None):
+    """tdq_w4a4_linear_pow2: the linear layer for power-of-two activation steps.  Returns y [M, O]."""
+    _need_cuda(xcodes, xscale, wcodes, wscale, bias)
+    M, half = xcodes.shape
+    I_pad = half * 2
+    O = wcodes.shape[0]
+    if y is None:
+        y = torch.empty((M, O), dtype=out_dtype, device=xcodes.device)
+    if workspace is None:
+        workspace = linear_workspace(M, I_pad, O, g, xcodes.device)
+    _check(_lib.tdq_w4a4_linear_pow2(_ptr(xcodes), _ptr(xscale), _ptr(wcodes), _ptr(wscale), _ptr(bias), M, I_pad, O, g,
+                                     _ptr(y), _dtype_id(y), y.stride(0) if M > 0 else O, _ptr(workspace),
+                                     workspace.numel(), _stream(xcodes)), "tdq_w4a4_linear_pow2")
     return y
 
 

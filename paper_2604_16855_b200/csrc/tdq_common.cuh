@@ -25,7 +25,7 @@ extern std::atomic<uint64_t> g_launch_count;
 
 // The linear layer with either source of its A operand.  fx == nullptr: activation codes and
 // scales from memory (tdq_w4a4_linear).  Otherwise the activations themselves, quantized by the
-// GEMM's own producer; xcodes and xscale are ignored.
+// GEMM's own producer; xcodes and xscale are ignored.  pow2_steps != 0: tdq_w4a4_linear_pow2.
 struct FusedSrc {
     const void* x;
     int64_t row_stride;   // elements
@@ -36,7 +36,7 @@ struct FusedSrc {
 tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* xscale, const uint8_t* wcodes,
                        const float* wscale, const float* bias, int64_t M, int64_t I_pad, int64_t O, int32_t group_size,
                        void* y, tdq_dtype y_dtype, int64_t y_row_stride, int32_t* acc_debug, void* workspace,
-                       size_t workspace_bytes, void* cuda_stream);
+                       size_t workspace_bytes, void* cuda_stream, int pow2_steps);
 // Argument checks of the quantizer and its fast-path conditions (tdq_quantize_act.cu).
 tdq_status check_act_args(const void* x, tdq_dtype dt, int64_t B, int64_t N, int64_t C, int64_t stride,
                           const tdq_act_params* p);

@@ -26,5 +26,5 @@ extern "C" tdq_status tdq_quant_linear_fused(const void* x, tdq_dtype x_dtype, i
     fx.seven_tau = 7.0f * p->tau;
     fx.flags = p->flags;
     return linear_impl(&fx, nullptr, nullptr, wcodes, wscale, bias, B * N, C, O, 32, y, y_dtype, y_row_stride, nullptr,
-                       workspace, workspace_bytes, cuda_stream);
+                       workspace, workspace_bytes, cuda_stream, 0);
 }

@@ -428,6 +428,81 @@ __global__ void __launch_bounds__(kExpandThreads) expand_kernel(ExpandArgs a) {
     }
 }
 
+// Power-of-two steps (tdq_w4a4_linear_pow2): the group scale goes into the operand.  With every step of a
+// row a power of two, Delta[m,k] = 2^(e_m + s), a code is stored as the E4M3 value q * 2^(s - 9), where
+// e_m is the row's largest step exponent minus 14, so s runs over 0..14: |q| <= 8 has at most three
+// significant bits and E4M3 four, and q * 2^(s-9) lies between 2^-9 (the smallest subnormal) and 256, so
+// the byte is exact.  Steps more than 2^14 below the row's largest have s < 0 and lose their low bits
+// (truncated).  The whole contraction then accumulates in one fp32 accumulator and the row needs one
+// scale, 2^e_m, in the epilogue.
+__device__ __forceinline__ uint32_t pow2_byte(uint32_t nib, int s) {
+    const uint32_t neg = nib & 8u;
+    const uint32_t mag = neg ? 16u - nib : nib;            // |q| in 0..8
+    const uint32_t t = s >= 0 ? mag << s : mag >> min(-s, 31);
+    uint32_t b;
+    if (t < 8u) {
+        b = t;                                             // subnormal: t * 2^-9
+    } else {
+        const int p = 31 - __clz(t);                       // t = 1.m * 2^p
+        b = ((uint32_t)(p - 2) << 3) | ((t >> (p - 3)) & 7u);
+    }
+    return b | (neg << 4);                                 // sign bit 7
+}
+
+__global__ void __launch_bounds__(kExpandThreads) expand_pow2_kernel(ExpandArgs a, int32_t act_steps_per_grp, int32_t act_Kg) {
+    const int piece = blockIdx.x;
+    if (piece == 0 && threadIdx.x < 4) a.status[threadIdx.x] = 0u;
+    const int blk = piece / a.n_chunks, kc = piece % a.n_chunks;
+    const int r = threadIdx.x >> 2;
+    const int ks = kc * kChunk + (threadIdx.x & 3);
+    if (ks >= a.n_steps) return;
+    const bool is_a = blk < a.tiles_m;
+    const int tile = is_a ? blk : blk - a.tiles_m;
+    const int64_t row = (int64_t)tile * 128 + r;
+    const int64_t rows = is_a ? a.M : a.O;
+    const uint8_t* src = is_a ? a.xcodes : a.wcodes;
+    uint4 p = make_uint4(0, 0, 0, 0);
+    if (row < rows) p = __ldg(reinterpret_cast<const uint4*>(src + row * a.row_bytes + (int64_t)ks * 16));
+    uint4 c0, c1;
+    if (!is_a) {
+        expand8<false>(p.x, c0.x, c0.y);
+        expand8<false>(p.y, c0.z, c0.w);
+        expand8<false>(p.z, c1.x, c1.y);
+        expand8<false>(p.w, c1.z, c1.w);
+    } else {
+        int s = 0;
+        uint32_t row_scale = 0u;                           // bits of 2^e_m
+        if (row < rows) {
+            const float* sc = a.xscale + row * act_Kg;
+            uint32_t emax = 0u, bad = 0u;
+            for (int k = 0; k < act_Kg; ++k) {
+                const uint32_t bits = __float_as_uint(__ldg(sc + k));
+                emax = max(emax, bits >> 23);
+                bad |= bits & 0x807fffffu;                 // a mantissa or a sign: not a power of two
+            }
+            if (bad) atomicCAS(a.status, 0u, 11u | ((uint32_t)tile << 8));   // reported through the status word
+            const int e_m = (int)emax - 14;
+            s = (int)(__float_as_uint(__ldg(sc + ks / act_steps_per_grp)) >> 23) - e_m;
+            row_scale = e_m > 0 ? (uint32_t)e_m << 23 : 0u;
+        }
+        uint32_t w[8];
+        const uint32_t pw[4] = {p.x, p.y, p.z, p.w};
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {                      // four nibbles -> four bytes
+            const uint32_t h = (pw[i >> 1] >> (16 * (i & 1))) & 0xffffu;
+            w[i] = pow2_byte(h & 15u, s) | (pow2_byte((h >> 4) & 15u, s) << 8) | (pow2_byte((h >> 8) & 15u, s) << 16) |
+                   (pow2_byte(h >> 12, s) << 24);
+        }
+        c0 = make_uint4(w[0], w[1], w[2], w[3]);
+        c1 = make_uint4(w[4], w[5], w[6], w[7]);
+        if (ks == 0) reinterpret_cast<uint32_t*>(a.s_blocks + (int64_t)tile * kScaleBlock)[r] = row_scale;
+    }
+    uint8_t* dst = (is_a ? a.a_blocks : a.b_blocks) + ((int64_t)tile * a.n_steps + ks) * kBlock;
+    const int off = (r >> 3) * 256 + (r & 7) * 16;
+    *reinterpret_cast<uint4*>(dst + off) = c0;
+    *reinterpret_cast<uint4*>(dst + off + 128) = c1;
+}
+
 // ------------------------------------------------------------------------------------------
 // kernel 2: the GEMM
 
@@ -1112,8 +1187,9 @@ namespace tdq {
 tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* xscale, const uint8_t* wcodes,
                        const float* wscale, const float* bias, int64_t M, int64_t I_pad, int64_t O, int32_t group_size,
                        void* y, tdq_dtype y_dtype, int64_t y_row_stride, int32_t* acc_debug, void* workspace,
-                       size_t workspace_bytes, void* cuda_stream) {
+                       size_t workspace_bytes, void* cuda_stream, int pow2_steps) {
     if (!fx && (!xcodes || !xscale)) return TDQ_ERR_INVALID_ARG;
+    if (pow2_steps && (fx || acc_debug)) return TDQ_ERR_UNSUPPORTED;
     if (fx && (!fx->x || group_size != 32 || acc_debug)) return TDQ_ERR_UNSUPPORTED;
     if (!wcodes || !wscale || !y) return TDQ_ERR_INVALID_ARG;
     if (M < 0 || O <= 0 || I_pad <= 0 || y_row_stride < O) return TDQ_ERR_INVALID_ARG;
@@ -1121,6 +1197,13 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
     if (group_size <= 0 || I_pad % group_size) return TDQ_ERR_INVALID_ARG;
     if (group_size % 32 || group_size > 4096) return TDQ_ERR_UNSUPPORTED;
     if (I_pad / 2 > INT32_MAX) return TDQ_ERR_INVALID_ARG;
+    // power-of-two steps: the activation groups only matter to the operand encoding; the kernel sees one
+    // group that spans the whole contraction
+    const int32_t act_group = group_size;
+    if (pow2_steps) {
+        if (I_pad > INT32_MAX) return TDQ_ERR_UNSUPPORTED;
+        group_size = (int32_t)I_pad;
+    }
     Plan p;
     if (!make_plan(M, I_pad, O, group_size, 148, p)) return TDQ_ERR_UNSUPPORTED;
     if (!workspace || workspace_bytes < kWorkspaceHeader + p.a_bytes + p.b_bytes + p.s_bytes) return TDQ_ERR_WORKSPACE;
@@ -1135,7 +1218,9 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
     if (fx && !p.a_resident) return TDQ_ERR_UNSUPPORTED;   // the fused producer writes a whole row block's A into shared memory
 
     uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
-    const bool i8 = group_size > 32;   // several instructions chain into one slot: keep the integer accumulator
+    // several instructions chain into one slot: keep the integer accumulator (the power-of-two variant
+    // accumulates scaled values, which only the fp32 accumulator can hold)
+    const bool i8 = group_size > 32 && !pow2_steps;
 
     ExpandArgs e;
     e.xcodes = xcodes; e.xscale = xscale; e.wcodes = wcodes;
@@ -1151,7 +1236,7 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
     // workspace; its promotion warps do that at the start of an item, though, with the tensor core idle,
     // so it only pays when an item carries much more work than its own unpacking.
     const int64_t steps_per_item = (p.tiles_n + p.n_parts - 1) / p.n_parts * (int64_t)p.n_steps;
-    const bool unpack_a = !fx && p.a_resident && steps_per_item >= 256;
+    const bool unpack_a = !fx && !pow2_steps && p.a_resident && steps_per_item >= 256;
     e.tiles_m = (fx || unpack_a) ? 0 : (int32_t)p.tiles_m;   // then only the weights are expanded here
     e.tiles_n = (int32_t)p.tiles_n;
     e.status = reinterpret_cast<uint32_t*>(workspace);
@@ -1197,7 +1282,9 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
         return TDQ_ERR_CUDA;
 
     const unsigned pieces = (unsigned)((e.tiles_m + e.tiles_n) * p.n_chunks);
-    if (i8)
+    if (pow2_steps)
+        expand_pow2_kernel<<<pieces, kExpandThreads, 0, stream>>>(e, act_group / 32, (int32_t)(I_pad / act_group));
+    else if (i8)
         expand_kernel<true><<<pieces, kExpandThreads, 0, stream>>>(e);
     else
         expand_kernel<false><<<pieces, kExpandThreads, 0, stream>>>(e);
@@ -1220,7 +1307,15 @@ extern "C" tdq_status tdq_w4a4_linear(const uint8_t* xcodes, const float* xscale
                                       int32_t* acc_debug, void* workspace, size_t workspace_bytes,
                                       void* cuda_stream) {
     return linear_impl(nullptr, xcodes, xscale, wcodes, wscale, bias, M, I_pad, O, group_size, y, y_dtype, y_row_stride,
-                       acc_debug, workspace, workspace_bytes, cuda_stream);
+                       acc_debug, workspace, workspace_bytes, cuda_stream, 0);
+}
+
+extern "C" tdq_status tdq_w4a4_linear_pow2(const uint8_t* xcodes, const float* xscale, const uint8_t* wcodes,
+                                           const float* wscale, const float* bias, int64_t M, int64_t I_pad, int64_t O,
+                                           int32_t group_size, void* y, tdq_dtype y_dtype, int64_t y_row_stride,
+                                           void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return linear_impl(nullptr, xcodes, xscale, wcodes, wscale, bias, M, I_pad, O, group_size, y, y_dtype, y_row_stride,
+                       nullptr, workspace, workspace_bytes, cuda_stream, 1);
 }
 
 extern "C" tdq_status tdq_workspace_status(const void* workspace, void* cuda_stream, uint32_t* detail) {

@@ -387,3 +387,56 @@ def test_power_of_two_steps_match_oracle(tdq, idx, bf16, g):
     np.testing.assert_array_equal(codes, ref["codes"])
     np.testing.assert_array_equal(scale, ref["scale"])
     assert np.all(np.frexp(scale.astype(np.float64))[0] == 0.5)
+
+
+def _pow2_case(tdq, x_np, bf16, w_np, g=32, bias=None, out_dtype=torch.float32):
+    xa = oracle.quantize_act(x_np, g=g, flags=7)
+    wq = oracle.quantize_weight(w_np, pad_to=g)
+    wsp = tdq.linear_workspace(xa["codes"].shape[0], xa["codes"].shape[1] * 2, w_np.shape[0], g, "cuda")
+    y = tdq.w4a4_linear_pow2(to_cuda(xa["codes"]), to_cuda(xa["scale"]), to_cuda(wq["codes"]), to_cuda(wq["scale"]),
+                             None if bias is None else to_cuda(bias), g=g, out_dtype=out_dtype, workspace=wsp)
+    st, detail = tdq.workspace_status(wsp)
+    assert st == tdq.OK, "status 0x%x" % detail
+    ref = oracle.w4a4_linear(xa["codes"], xa["scale"], wq["codes"], wq["scale"], bias=bias, g=g)
+    return y.float().cpu().numpy(), ref, xa
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("idx,rows,g", [(1, None, 32), (2, 3000, 32), (3, 1500, 32), (3, 700, 64), (4, 300, 32)])
+def test_power_of_two_linear_matches_the_exact_layer(tdq, idx, rows, g):
+    case = si.config(idx)
+    x = case.x.reshape(-1, case.C)
+    if rows:
+        x = x[:rows]
+    bias = np.linspace(-0.02, 0.02, case.O).astype(np.float32) if idx == 3 else None
+    y, ref, xa = _pow2_case(tdq, x, case.x_is_bf16, case.w, g=g, bias=bias)
+    # the steps of a row span fewer than 15 binades here, so nothing is truncated; what remains is the
+    # binary32 accumulation of C products in the tensor core's order
+    spread = np.log2(xa["scale"].max(axis=1) / xa["scale"].min(axis=1)).max()
+    assert spread <= 14
+    worst, strict = compare_y(y, ref, case.C)
+    assert strict > 0.99
+
+
+@pytest.mark.gpu
+def test_power_of_two_linear_truncation_bound_bf16_output_and_bad_scales(tdq):
+    rng = np.random.RandomState(9)
+    M, C, O = 200, 128, 96
+    x = rng.normal(size=(M, C)).astype(np.float32)
+    x[:, 32:64] *= 1e-6                                    # one group 2^20 below the others: truncated
+    w = (rng.normal(size=(O, C)) * 0.02).astype(np.float32)
+    y, ref, xa = _pow2_case(tdq, x, False, w)
+    wq = oracle.quantize_weight(w)
+    big = xa["scale"].max(axis=1, keepdims=True).astype(np.float64)
+    bound = 32 * 8 * wq["scale"].astype(np.float64)[None, :] * big * 2.0 ** -14      # 32 truncated elements, |q_w| <= 8
+    tol = np.maximum(1e-5 * np.abs(ref["y_d"]), (C + 2) * 2.0 ** -24 * ref["t_abs"]) + bound
+    assert np.all(np.abs(y - ref["y_d"]) <= tol)
+    # bf16 output and a ragged shape
+    yb, refb, _ = _pow2_case(tdq, x[:131], False, w[:70], out_dtype=torch.bfloat16)
+    assert np.all(np.abs(yb - refb["y_d"]) <= 2.0 ** -8 * np.abs(refb["y_d"]) + bound[:131, :70] + 1e-6)
+    # a step that is not a power of two is reported
+    xa2 = oracle.quantize_act(x)                           # the paper's steps
+    wsp = tdq.linear_workspace(M, C, O, 32, "cuda")
+    tdq.w4a4_linear_pow2(to_cuda(xa2["codes"]), to_cuda(xa2["scale"]), to_cuda(wq["codes"]), to_cuda(wq["scale"]), workspace=wsp)
+    st, detail = tdq.workspace_status(wsp)
+    assert st != tdq.OK and (detail & 0xff) == 11
