@@ -270,6 +270,29 @@ __device__ __forceinline__ void mma_issue_if(uint32_t on, uint32_t d_tmem, uint3
             ::"r"(d_tmem), "r"(adesc_lo), "r"(bdesc_lo), "r"(kIdescF8), "r"(accumulate), "r"(on), "r"(kDescHi)
             : "memory");
 }
+// Four instructions on consecutive K-steps of the same accumulator (operand blocks 4096 bytes apart): the
+// predicates and the descriptors are built once, the descriptors move by an add.
+template <bool I8>
+__device__ __forceinline__ void mma_issue4_if(uint32_t on, uint32_t d_tmem, uint32_t adesc_lo, uint32_t bdesc_lo,
+                                              uint32_t accumulate_first) {
+#define TDQ_MMA4(KIND, IDESC)                                                                       \
+    asm volatile(                                                                                   \
+        "{\n\t.reg .pred p, q, t;\n\t.reg .b64 da, db;\n\t"                                        \
+        "setp.ne.b32 p, %4, 0;\n\tsetp.ne.b32 q, %5, 0;\n\tsetp.eq.b32 t, 0, 0;\n\t"                 \
+        "mov.b64 da, {%1, %6};\n\tmov.b64 db, {%2, %6};\n\t"                                        \
+        "@q tcgen05.mma.cta_group::1.kind::" KIND " [%0], da, db, %3, p;\n\t"                        \
+        "add.s64 da, da, 256;\n\tadd.s64 db, db, 256;\n\t"                                          \
+        "@q tcgen05.mma.cta_group::1.kind::" KIND " [%0], da, db, %3, t;\n\t"                        \
+        "add.s64 da, da, 256;\n\tadd.s64 db, db, 256;\n\t"                                          \
+        "@q tcgen05.mma.cta_group::1.kind::" KIND " [%0], da, db, %3, t;\n\t"                        \
+        "add.s64 da, da, 256;\n\tadd.s64 db, db, 256;\n\t"                                          \
+        "@q tcgen05.mma.cta_group::1.kind::" KIND " [%0], da, db, %3, t;\n\t}"                       \
+        ::"r"(d_tmem), "r"(adesc_lo), "r"(bdesc_lo), "r"(IDESC), "r"(accumulate_first), "r"(on), "r"(kDescHi) \
+        : "memory")
+    if (I8) TDQ_MMA4("i8", kIdescI8);
+    else TDQ_MMA4("f8f6f4", kIdescF8);
+#undef TDQ_MMA4
+}
 __device__ __forceinline__ void mma_commit_if(uint32_t on, uint32_t bar_s) {
     asm volatile(
         "{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
@@ -707,10 +730,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                                 }
                                 tc_fence_after();
                                 const uint32_t d_tmem = tmem_base + slot * kBN;
-                                mma_issue_if<I8>(lane0, d_tmem, a_lo, b_lo, sub == 0 ? 0u : 1u);
-                                mma_issue_if<I8>(lane0, d_tmem, a_lo + 1 * (kBlock >> 4), b_lo + 1 * (kBlock >> 4), 1u);
-                                mma_issue_if<I8>(lane0, d_tmem, a_lo + 2 * (kBlock >> 4), b_lo + 2 * (kBlock >> 4), 1u);
-                                mma_issue_if<I8>(lane0, d_tmem, a_lo + 3 * (kBlock >> 4), b_lo + 3 * (kBlock >> 4), 1u);
+                                static_assert((kBlock >> 4) == 256, "mma_issue4_if moves the descriptors by 256");
+                                mma_issue4_if<I8>(lane0, d_tmem, a_lo, b_lo, sub == 0 ? 0u : 1u);
                                 sub += kChunk;
                                 if (sub == spg) {
                                     sub = 0;
