@@ -425,6 +425,7 @@ def run_tdq(args):
     q_iso_ms = l_iso_ms = None
     q_switch_ms = None
     q_nchw = None
+    pow2 = None
     if world == 1 and not args.no_extras:
         # each kernel on its own, launched back to back from a graph over rotating buffers: no other
         # kernel and no event node between two launches (the in-step figures above include those gaps)
@@ -455,6 +456,13 @@ def run_tdq(args):
         del fm, fcodes, fscale
         l_iso_ms = time_graph(lambda i: tdq.w4a4_linear(codes[i % nsets], scales[i % nsets], wcodes, wscale, y=ys[i % nsets],
                                                         workspace=wsp), 8 * nsets)
+        # the power-of-two step variant (not the paper's quantizer): its quantizer and its linear layer
+        p2 = tdq.act_params(flags=tdq.ENABLE_C1 | tdq.ENABLE_C2 | tdq.POW2_STEP)
+        tdq.quantize_act(xs[0], p2, codes=codes[0], scale=scales[0])
+        pl_ms = time_graph(lambda i: tdq.w4a4_linear_pow2(codes[0], scales[0], wcodes, wscale, y=ys[i % nsets], workspace=wsp),
+                           8 * nsets)
+        pow2 = dict(name="tdq_w4a4_linear_pow2", ms=pl_ms, tops=2.0 * M * C * O / (pl_ms * 1e-3) / 1e12,
+                    gbs=linear_bytes(M, C, O) / (pl_ms * 1e-3) / 1e9)
         fused = fused_leg(tdq, xs, wcodes, wscale, ys, wsp, M, C, O, esize)
         del xs, codes, scales, ys
         torch.cuda.empty_cache()
@@ -504,7 +512,7 @@ def run_tdq(args):
                                cache="rotating %d buffer sets, %.0f MB per step (L2 is 126 MB)" % (nsets, step_bytes / 1e6),
                                launch=("CUDA graph of %d steps, replayed %d times" % (G, args.steps // G)) if G else "eager",
                                parallelism="rows sharded, %d replica(s)" % world),
-                   kernels=dict(quantize_act=q_kernel, quantize_act_nchw=q_nchw, w4a4_linear=l_kernel, fused=fused, sweep_cfg5=sweep,
+                   kernels=dict(quantize_act=q_kernel, quantize_act_nchw=q_nchw, w4a4_linear=l_kernel, w4a4_linear_pow2=pow2, fused=fused, sweep_cfg5=sweep,
                                 step_tokens_per_s=world * M * K / (total_ms * 1e-3)),
                    roofline=roof, clocks=clocks, gpu_launches=int(launches),
                    e2e=dict(value=e2e_value, unit="GB/s", ms_per_step=e2e_ms / e2e_steps,
