@@ -112,6 +112,8 @@ struct LinArgs {
     int32_t a_resident;        // the item's whole A block stays in shared memory
     int32_t n_stages;
     uint32_t ring_off, stage_bytes, staging_off;   // shared-memory carve-up
+    uint32_t staging_bytes;    // all sixteen strips: 64 KB, or 32 KB when a strip holds 32 rows of 64 bytes
+    int32_t half_strips;       // fp32 output written in two passes of 16 columns through 64-byte strip rows
     uint32_t ibuf_bytes;       // one item buffer: the item's scales, then its A blocks if resident
     int32_t n_ibuf;            // item buffers (1..kMaxItemBufs): the producer runs that many items ahead
     void* y;
@@ -791,10 +793,11 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
         constexpr int esz = YBF16 ? 2 : 4;
         constexpr uint32_t kRowBytes = kCols * esz;   // one row of the strip
         const uint32_t strips_s = (sm_s + a.staging_off + 1023u) & ~1023u;   // the swizzle pattern repeats every 1024 bytes
-        const uint32_t strip_w = strips_s + (uint32_t)pw * (32 * kStripBytes);
-        const uint32_t strip_row = strip_w + (uint32_t)lane * kRowBytes;
-        const uint32_t swz = YBF16 ? (((uint32_t)lane >> 1) & 3u) : ((uint32_t)lane & 7u);   // chunk c sits at c ^ swz
-        const uint32_t wsb_s = strips_s + kStagingBytes + (uint32_t)pw * 256;
+        const bool narrow = YBF16 || a.half_strips;   // 64-byte strip rows
+        const uint32_t strip_w = strips_s + (uint32_t)pw * (a.staging_bytes / kPromoWarps);
+        const uint32_t strip_row = strip_w + (uint32_t)lane * (narrow ? 64u : 128u);
+        const uint32_t swz = narrow ? (((uint32_t)lane >> 1) & 3u) : ((uint32_t)lane & 7u);   // chunk c sits at c ^ swz
+        const uint32_t wsb_s = strips_s + a.staging_bytes + (uint32_t)pw * 256;
         uint32_t ib = 0, iu = 0;                      // item buffer and its phase
         uint32_t my_scale_s = ibuf_s + (uint32_t)row * 4;   // this row's scales in the current item buffer
 
@@ -911,7 +914,42 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
             store_pending = false;
         };
         // y = (s_o * 2^e) * sum + bias for the tile that just finished, then on to the next tile
+        // The same epilogue in two passes of 16 columns (fp32 output of wide groups, where the promotion warps
+        // have time to spare): a strip is 32 rows of 64 bytes, half the shared memory, and the ring gets the
+        // other half as two more stages.  The second pass waits until the engine has read the first.
+        auto finish_tile_half = [&]() {
+            float* wsb = reinterpret_cast<float*>(smem_raw + (wsb_s - sm_s));
+            wsb[lane] = __fmul_rn(w0, a.out_scale);
+            wsb[32 + lane] = b0;
+            uint8_t* strip = smem_raw + (strip_row - sm_s);
+            const int64_t m0 = (int64_t)mt * kBM + quarter * 32;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                if (lane == 0) bulk_wait_group_read0();      // the previous pass's store has read the strip
+                __syncwarp();
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {
+                    const int j = 4 * h + jj;
+                    float o0, o1, o2, o3;
+                    unpack2(yacc[2 * j], o0, o1);
+                    unpack2(yacc[2 * j + 1], o2, o3);
+                    const float4 s4 = reinterpret_cast<const float4*>(wsb)[j], b4 = reinterpret_cast<const float4*>(wsb + 32)[j];
+                    *reinterpret_cast<float4*>(strip + (((uint32_t)jj ^ swz) << 4)) =
+                        make_float4(__fmaf_rn(s4.x, o0, b4.x), __fmaf_rn(s4.y, o1, b4.y), __fmaf_rn(s4.z, o2, b4.z),
+                                    __fmaf_rn(s4.w, o3, b4.w));
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0 && m0 < a.M && n0 + 16 * h < a.O) {
+                    tma_store_2d(&ymap, strip_w, (int32_t)n0 + 16 * h, (int32_t)m0);
+                    bulk_commit_group();
+                }
+            }
+        };
         auto finish_tile = [&]() {
+            if (!YBF16 && a.half_strips) {
+                finish_tile_half();
+            } else {
             if (store_pending) issue_store();            // a short tile: the previous store is still waiting for its turn
             if (lane == 0) bulk_wait_group_read0();      // the previous tile's store has read the strip
             float* wsb = reinterpret_cast<float*>(smem_raw + (wsb_s - sm_s));
@@ -967,6 +1005,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                     }
                 }
                 __syncwarp();     // the strip may be overwritten by the next tile
+            }
             }
             // next tile, next item
             if (++nt == nt_end) {
@@ -1097,7 +1136,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
 typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                       const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                       CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-bool encode_y_map(CUtensorMap* map, void* y, bool bf16, int64_t M, int64_t O, int64_t y_row_stride) {
+bool encode_y_map(CUtensorMap* map, void* y, bool bf16, int64_t M, int64_t O, int64_t y_row_stride, int box_cols) {
     static const TensorMapEncodeFn encode = [] {
         void* fn = nullptr;
         cudaDriverEntryPointQueryResult res;
@@ -1110,10 +1149,11 @@ bool encode_y_map(CUtensorMap* map, void* y, bool bf16, int64_t M, int64_t O, in
     const cuuint64_t esz = bf16 ? 2 : 4;
     const cuuint64_t dims[2] = {(cuuint64_t)O, (cuuint64_t)M};
     const cuuint64_t strides[1] = {(cuuint64_t)y_row_stride * esz};
-    const cuuint32_t box[2] = {(cuuint32_t)kCols, 32u};
+    const cuuint32_t box[2] = {(cuuint32_t)box_cols, 32u};
+    const bool rows64 = (size_t)box_cols * esz == 64;   // 64-byte strip rows (else 128)
     const cuuint32_t elem_strides[2] = {1u, 1u};
     return encode(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, y, dims, strides, box,
-                  elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, bf16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                  elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, rows64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
                   CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -1128,7 +1168,7 @@ struct Plan {
 constexpr size_t kWorkspaceHeader = 256;   // status word, then the blocks
 
 // false: sizes out of range, or the problem's scales plus two ring stages do not fit in shared memory
-bool make_plan(int64_t M, int64_t I_pad, int64_t O, int32_t g, int n_sm, Plan& p) {
+bool make_plan(int64_t M, int64_t I_pad, int64_t O, int32_t g, int n_sm, Plan& p, int64_t staging_bytes = kStagingBytes) {
     p.tiles_m = (M + kBM - 1) / kBM;
     p.tiles_n = (O + kBN - 1) / kBN;
     if (p.tiles_m > INT32_MAX / 4096 || p.tiles_n > INT32_MAX / 4096 || I_pad / 32 > INT32_MAX / 8) return false;
@@ -1140,7 +1180,7 @@ bool make_plan(int64_t M, int64_t I_pad, int64_t O, int32_t g, int n_sm, Plan& p
     p.s_bytes = (size_t)p.tiles_m * p.Kg * kScaleBlock;
     // shared memory: control, the item's scales, [resident A], ring, output strips, channel scales
     const int64_t scales = (int64_t)p.Kg * kScaleBlock;
-    const int64_t fixed = 1024 + kCtrlBytes + scales + kStagingBytes + kWsbBytes;   // 1024: the strips start on a 1 KB boundary
+    const int64_t fixed = 1024 + kCtrlBytes + scales + staging_bytes + kWsbBytes;   // 1024: the strips start on a 1 KB boundary
     const int64_t a_res = (int64_t)p.n_steps * kBlock;
     const int64_t stage_b = (int64_t)kChunk * kBlock, stage_ab = 2 * stage_b;
     const int64_t stages_res = (kSmemLimit - fixed - a_res) / stage_b;
@@ -1165,7 +1205,7 @@ bool make_plan(int64_t M, int64_t I_pad, int64_t O, int32_t g, int n_sm, Plan& p
     }
     p.ring_off = (uint32_t)kCtrlBytes + (uint32_t)p.n_ibuf * p.ibuf_bytes;
     p.staging_off = p.ring_off + (uint32_t)p.n_stages * p.stage_bytes;
-    p.smem_bytes = p.staging_off + 1024 + kStagingBytes + kWsbBytes;
+    p.smem_bytes = p.staging_off + 1024 + (uint32_t)staging_bytes + kWsbBytes;
     // split the column tiles of a row block into parts so that the items fill the SMs evenly
     int best = 1;
     int64_t best_cost = INT64_MAX;
@@ -1235,7 +1275,15 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
     const int n_sm = sm_count();
     if (n_sm <= 0) return TDQ_ERR_CUDA;
-    if (!make_plan(M, I_pad, O, group_size, n_sm, p)) return TDQ_ERR_UNSUPPORTED;
+    // Output strips: 64-byte rows (32 KB in all) for bf16 output, and for fp32 output of wide groups, which is
+    // then written in two passes of 16 columns; the ring gets the other 32 KB.  Both need the bulk tensor store.
+    const int64_t y_esz = y_dtype == TDQ_BF16 ? 2 : 4;
+    const bool y_tma = reinterpret_cast<uintptr_t>(y) % 16 == 0 && (y_row_stride * y_esz) % 16 == 0 && O <= INT32_MAX &&
+                       M <= INT32_MAX;
+    const bool half_strips = y_tma && y_dtype == TDQ_F32 && !fx && !acc_debug && group_size >= 128;
+    const bool narrow_strips = y_tma && (y_dtype == TDQ_BF16 || half_strips);
+    const int64_t staging_bytes = narrow_strips ? kStagingBytes / 2 : kStagingBytes;
+    if (!make_plan(M, I_pad, O, group_size, n_sm, p, staging_bytes)) return TDQ_ERR_UNSUPPORTED;
     if (fx && !p.a_resident) return TDQ_ERR_UNSUPPORTED;   // the fused producer writes a whole row block's A into shared memory
 
     uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
@@ -1279,9 +1327,12 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
     CUtensorMap ymap;
     memset(&ymap, 0, sizeof(ymap));
     a.tma_ok = 0;
-    if (reinterpret_cast<uintptr_t>(y) % 16 == 0 && (y_row_stride * esz) % 16 == 0 && O <= INT32_MAX && M <= INT32_MAX &&
-        encode_y_map(&ymap, y, y_dtype == TDQ_BF16, M, O, y_row_stride))
+    if (y_tma && encode_y_map(&ymap, y, y_dtype == TDQ_BF16, M, O, y_row_stride, half_strips ? kCols / 2 : kCols))
         a.tma_ok = 1;
+    else if (narrow_strips)
+        return TDQ_ERR_CUDA;   // the plan counted on the tensor store
+    a.staging_bytes = (uint32_t)staging_bytes;
+    a.half_strips = half_strips ? 1 : 0;
     a.out_scale = i8 ? 0.00390625f : 262144.0f;
     a.xcodes = xcodes; a.xscale = xscale; a.row_bytes = e.row_bytes; a.unpack_a = unpack_a ? 1 : 0;
     a.x = fx ? fx->x : nullptr;
