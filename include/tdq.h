@@ -195,9 +195,15 @@ tdq_status tdq_quant_linear_fused(const void* x, tdq_dtype x_dtype, int64_t B, i
 
 /*
  * The two-kernel path with HOST input and output: copies x_host to x_dev, runs
- * tdq_quantize_act and tdq_w4a4_linear, copies y_dev to y_host, all on cuda_stream.
+ * tdq_quantize_act and tdq_w4a4_linear, copies y_dev to y_host.  The rows go through in up to
+ * eight chunks: the kernels run on cuda_stream, the copies on two side streams of the library
+ * (created on the first call on a device and tied to cuda_stream by events), so that the
+ * copy-out of one chunk overlaps the copy-in and the kernels of the next.  Work queued on
+ * cuda_stream after the call starts only when the last copy-out has finished.
  * x_host / y_host should be page-locked for the copies to be asynchronous.  The device
- * buffers are the caller's and sized as for the two calls (x_dev [B*N, C] dense).
+ * buffers are the caller's and sized as for the two calls (x_dev [B*N, C] dense).  The chunks
+ * share the workspace one after another, so tdq_workspace_status afterwards speaks for the last
+ * chunk only.  Not for concurrent use from several host threads on one device.
  */
 tdq_status tdq_quant_linear_host(const void* x_host /* HOST */, tdq_dtype x_dtype, int64_t B, int64_t N,
                                  int64_t C, const tdq_act_params* p /* HOST */, const uint8_t* wcodes,

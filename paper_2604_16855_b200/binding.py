@@ -271,6 +271,31 @@ def quant_linear_fused(x, wcodes, wscale, bias=None, params: ActParams | None = 
     return y
 
 
+def quant_linear_host(x_host: torch.Tensor, wcodes, wscale, bias=None, params: ActParams | None = None, *,
+                      out_dtype=torch.float32, y_host=None, device="cuda"):
+    """tdq_quant_linear_host: x_host [M, C] (CPU, ideally pinned) in, y_host [M, O] (CPU) out.  The device buffers
+    the call needs are allocated here.  Returns (y_host, workspace); synchronise the current stream before reading."""
+    _need_cuda(wcodes, wscale, bias)
+    p = params or default_act_params()
+    M, C = x_host.shape
+    O = wcodes.shape[0]
+    g = p.group_size
+    I_pad = (C + g - 1) // g * g
+    dev = wcodes.device
+    x_dev = torch.empty((M, C), dtype=x_host.dtype, device=dev)
+    codes = torch.empty((M, I_pad // 2), dtype=torch.uint8, device=dev)
+    scale = torch.empty((M, I_pad // g), dtype=torch.float32, device=dev)
+    y_dev = torch.empty((M, O), dtype=out_dtype, device=dev)
+    if y_host is None:
+        y_host = torch.empty((M, O), dtype=out_dtype).pin_memory()
+    workspace = linear_workspace(M, I_pad, O, g, dev)
+    _check(_lib.tdq_quant_linear_host(_ptr(x_host), _dtype_id(x_host), 1, M, C, ctypes.byref(p), _ptr(wcodes), _ptr(wscale),
+                                      _ptr(bias), O, _ptr(y_host), _dtype_id(y_host), _ptr(x_dev), _ptr(codes), _ptr(scale),
+                                      _ptr(y_dev), _ptr(workspace), workspace.numel(), _stream(wcodes)),
+           "tdq_quant_linear_host")
+    return y_host, (workspace, x_dev, codes, scale, y_dev)
+
+
 def workspace_status(workspace: torch.Tensor):
     """(status, detail word) left by the last linear call that used this workspace; synchronises."""
     detail = ctypes.c_uint32(0)

@@ -19,6 +19,43 @@ extern "C" const char* tdq_status_string(tdq_status s) {
 
 extern "C" uint64_t tdq_kernel_launch_count(void) { return g_launch_count.load(std::memory_order_relaxed); }
 
+namespace {
+
+// Side streams and events of the host-buffer call, made once per process and device (the call is a
+// convenience for callers who hold host data; it is the one entry point that creates CUDA objects).
+constexpr int kHostChunks = 8;
+struct HostPipe {
+    cudaStream_t h2d = nullptr, d2h = nullptr;
+    cudaEvent_t start = nullptr, done = nullptr, in[kHostChunks] = {}, out[kHostChunks] = {};
+    bool ok = false;
+};
+HostPipe* host_pipe() {
+    static HostPipe pipes[64];
+    static std::atomic<int> guard{0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    HostPipe& p = pipes[dev];
+    if (p.ok) return &p;
+    while (guard.exchange(1, std::memory_order_acquire)) {}
+    if (!p.ok) {
+        bool good = cudaStreamCreateWithFlags(&p.h2d, cudaStreamNonBlocking) == cudaSuccess &&
+                    cudaStreamCreateWithFlags(&p.d2h, cudaStreamNonBlocking) == cudaSuccess &&
+                    cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming) == cudaSuccess &&
+                    cudaEventCreateWithFlags(&p.done, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; i < kHostChunks && good; ++i)
+            good = cudaEventCreateWithFlags(&p.in[i], cudaEventDisableTiming) == cudaSuccess &&
+                   cudaEventCreateWithFlags(&p.out[i], cudaEventDisableTiming) == cudaSuccess;
+        p.ok = good;
+    }
+    guard.store(0, std::memory_order_release);
+    return p.ok ? &p : nullptr;
+}
+
+}  // namespace
+
+// Rows go through in up to eight chunks so that the copy-out of one chunk (the long pole: y is eight
+// times the size of x at cfg4) overlaps the copy-in and the kernels of the next; kernels run on the
+// caller's stream, the copies on two side streams tied to it by events.
 extern "C" tdq_status tdq_quant_linear_host(const void* x_host, tdq_dtype x_dtype, int64_t B, int64_t N, int64_t C,
                                             const tdq_act_params* p, const uint8_t* wcodes, const float* wscale,
                                             const float* bias, int64_t O, void* y_host, tdq_dtype y_dtype,
@@ -32,16 +69,38 @@ extern "C" tdq_status tdq_quant_linear_host(const void* x_host, tdq_dtype x_dtyp
     const int64_t M = B * N;
     if (M == 0) return TDQ_OK;
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
-    const size_t xbytes = (size_t)M * C * (x_dtype == TDQ_BF16 ? 2 : 4);
-    const size_t ybytes = (size_t)M * O * (y_dtype == TDQ_BF16 ? 2 : 4);
-    if (cudaMemcpyAsync(x_dev, x_host, xbytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) return TDQ_ERR_CUDA;
-    tdq_status st = tdq_quantize_act(x_dev, x_dtype, B, N, C, C, p, codes_dev, scale_dev, nullptr, cuda_stream);
-    if (st != TDQ_OK) return st;
+    HostPipe* hp = host_pipe();
+    if (!hp) return TDQ_ERR_CUDA;
+    const int64_t xe = x_dtype == TDQ_BF16 ? 2 : 4, ye = y_dtype == TDQ_BF16 ? 2 : 4;
     const int64_t g = p->group_size;
-    const int64_t I_pad = (C + g - 1) / g * g;
-    st = tdq_w4a4_linear(codes_dev, scale_dev, wcodes, wscale, bias, M, I_pad, O, p->group_size, y_dev, y_dtype, O,
-                         nullptr, workspace, workspace_bytes, cuda_stream);
-    if (st != TDQ_OK) return st;
-    if (cudaMemcpyAsync(y_host, y_dev, ybytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return TDQ_ERR_CUDA;
+    const int64_t K = (C + g - 1) / g, I_pad = K * g;
+    int64_t rows_per = (M + kHostChunks - 1) / kHostChunks;
+    rows_per = (rows_per + 127) / 128 * 128;
+    if (cudaEventRecord(hp->start, stream) != cudaSuccess) return TDQ_ERR_CUDA;
+    if (cudaStreamWaitEvent(hp->h2d, hp->start, 0) != cudaSuccess || cudaStreamWaitEvent(hp->d2h, hp->start, 0) != cudaSuccess)
+        return TDQ_ERR_CUDA;
+    int chunk = 0;
+    for (int64_t m0 = 0; m0 < M; m0 += rows_per, ++chunk) {
+        const int64_t rows = M - m0 < rows_per ? M - m0 : rows_per;
+        const char* xh = reinterpret_cast<const char*>(x_host) + m0 * C * xe;
+        char* xd = reinterpret_cast<char*>(x_dev) + m0 * C * xe;
+        char* yd = reinterpret_cast<char*>(y_dev) + m0 * O * ye;
+        if (cudaMemcpyAsync(xd, xh, (size_t)(rows * C * xe), cudaMemcpyHostToDevice, hp->h2d) != cudaSuccess ||
+            cudaEventRecord(hp->in[chunk], hp->h2d) != cudaSuccess || cudaStreamWaitEvent(stream, hp->in[chunk], 0) != cudaSuccess)
+            return TDQ_ERR_CUDA;
+        tdq_status st = tdq_quantize_act(xd, x_dtype, 1, rows, C, C, p, codes_dev + m0 * (I_pad / 2), scale_dev + m0 * K, nullptr,
+                                         cuda_stream);
+        if (st != TDQ_OK) return st;
+        st = tdq_w4a4_linear(codes_dev + m0 * (I_pad / 2), scale_dev + m0 * K, wcodes, wscale, bias, rows, I_pad, O,
+                             p->group_size, yd, y_dtype, O, nullptr, workspace, workspace_bytes, cuda_stream);
+        if (st != TDQ_OK) return st;
+        if (cudaEventRecord(hp->out[chunk], stream) != cudaSuccess || cudaStreamWaitEvent(hp->d2h, hp->out[chunk], 0) != cudaSuccess ||
+            cudaMemcpyAsync(reinterpret_cast<char*>(y_host) + m0 * O * ye, yd, (size_t)(rows * O * ye), cudaMemcpyDeviceToHost,
+                            hp->d2h) != cudaSuccess)
+            return TDQ_ERR_CUDA;
+    }
+    // the caller's stream finishes only after the last copy-out
+    if (cudaEventRecord(hp->done, hp->d2h) != cudaSuccess || cudaStreamWaitEvent(stream, hp->done, 0) != cudaSuccess)
+        return TDQ_ERR_CUDA;
     return TDQ_OK;
 }

@@ -440,3 +440,26 @@ def test_power_of_two_linear_truncation_bound_bf16_output_and_bad_scales(tdq):
     tdq.w4a4_linear_pow2(to_cuda(xa2["codes"]), to_cuda(xa2["scale"]), to_cuda(wq["codes"]), to_cuda(wq["scale"]), workspace=wsp)
     st, detail = tdq.workspace_status(wsp)
     assert st != tdq.OK and (detail & 0xff) == 11
+
+
+# ------------------------------------------------------------------------------------------
+# host-buffer entry point (chunked copies overlapped with the kernels)
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("idx,rows", [(3, None), (2, 300), (1, None)])
+def test_host_buffer_call_equals_the_two_calls(tdq, idx, rows):
+    case = si.config(idx)
+    x = case.x.reshape(-1, case.C)
+    if rows:
+        x = x[:rows]
+    xt = to_cuda(x, bf16=case.x_is_bf16)
+    wc, ws = tdq.quantize_weight(to_cuda(case.w))
+    codes, scale = tdq.quantize_act(xt)
+    y_ref = tdq.w4a4_linear(codes, scale, wc, ws).cpu()
+    x_host = xt.cpu().pin_memory()
+    for _ in range(2):                       # twice: the side streams and events are reused
+        y_host, keep = tdq.quant_linear_host(x_host, wc, ws)
+        torch.cuda.current_stream().synchronize()
+        assert torch.equal(y_host.view(torch.int32), y_ref.view(torch.int32))
+        st, detail = tdq.workspace_status(keep[0])
+        assert st == tdq.OK
