@@ -463,3 +463,52 @@ def test_host_buffer_call_equals_the_two_calls(tdq, idx, rows):
         assert torch.equal(y_host.view(torch.int32), y_ref.view(torch.int32))
         st, detail = tdq.workspace_status(keep[0])
         assert st == tdq.OK
+
+
+# ------------------------------------------------------------------------------------------
+# seeded random shapes: every mode of the linear kernel (resident and streamed operands, several work
+# items per CTA, one to four item buffers, in-kernel unpacking, both strip layouts) on ragged sizes
+
+def _random_linear_shapes(n, seed=2024):
+    rng = np.random.RandomState(seed)
+    shapes = []
+    for _ in range(n):
+        C = int(rng.choice([32, 64, 96, 128, 256, 320, 512, 768, 832, 1024]))
+        gs = [g for g in (32, 64, 128, C) if C % g == 0]
+        g = int(gs[rng.randint(len(gs))])
+        M = int(rng.choice([1, 37, 128, 129, 300, 700, 1500]))
+        O = int(rng.choice([1, 8, 100, 128, 130, 384, 700]))
+        shapes.append((M, C, O, g, bool(rng.randint(2)), bool(rng.randint(2))))
+    return shapes
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("M,C,O,g,bf16_out,with_bias", _random_linear_shapes(40))
+def test_linear_random_shapes(tdq, M, C, O, g, bf16_out, with_bias):
+    rng = np.random.RandomState(M * 7 + C + O)
+    x = (rng.normal(size=(M, C)) * np.exp(rng.normal(0, 1.0, size=(M, 1)))).astype(np.float32)
+    w = (rng.normal(size=(O, C)) * 0.05).astype(np.float32)
+    bias = rng.normal(size=(O,)).astype(np.float32) * 0.1 if with_bias else None
+    y, ref = _linear_case(tdq, x, False, w, g=g, bias=bias, out_dtype=torch.bfloat16 if bf16_out else torch.float32,
+                          want_acc=not bf16_out and M * O * (C // g) < 4_000_000)
+    compare_y(y, ref, C // g, out_eps=2.0 ** -8 if bf16_out else 0.0)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("M,C,O,g,bf16_out,with_bias", [s for s in _random_linear_shapes(60, seed=7) if s[1] <= 768][:16])
+def test_fused_and_power_of_two_random_shapes(tdq, M, C, O, g, bf16_out, with_bias):
+    rng = np.random.RandomState(M + 3 * C + 5 * O)
+    x = (rng.normal(size=(M, C)) * np.exp(rng.normal(0, 1.0, size=(M, 1)))).astype(np.float32)
+    w = (rng.normal(size=(O, C)) * 0.05).astype(np.float32)
+    bias = rng.normal(size=(O,)).astype(np.float32) * 0.1 if with_bias else None
+    dt = torch.bfloat16 if bf16_out else torch.float32
+    xt, wc_ws = to_cuda(x), tdq.quantize_weight(to_cuda(w))
+    b = None if bias is None else to_cuda(bias)
+    # fused == the two calls, bit for bit (group size 32 is the fused path's)
+    codes, scale = tdq.quantize_act(xt)
+    y2 = tdq.w4a4_linear(codes, scale, *wc_ws, b, out_dtype=dt)
+    y1 = tdq.quant_linear_fused(xt, *wc_ws, b, out_dtype=dt)
+    assert torch.equal(y1.view(torch.int16 if bf16_out else torch.int32), y2.view(torch.int16 if bf16_out else torch.int32))
+    # power-of-two steps at the drawn group size against the exact layer's oracle
+    y, ref, _ = _pow2_case(tdq, x, False, w, g=g, bias=bias, out_dtype=dt)
+    compare_y(y, ref, C, out_eps=2.0 ** -8 if bf16_out else 0.0)
