@@ -475,8 +475,8 @@ __device__ __forceinline__ uint32_t pow2_byte(uint32_t nib, int s) {
 }
 
 __global__ void __launch_bounds__(kExpandThreads) expand_pow2_kernel(ExpandArgs a, int32_t act_steps_per_grp, int32_t act_Kg) {
+    // (the status words are cleared by the host before this kernel: it may itself report a bad scale)
     const int piece = blockIdx.x;
-    if (piece == 0 && threadIdx.x < 4) a.status[threadIdx.x] = 0u;
     const int blk = piece / a.n_chunks, kc = piece % a.n_chunks;
     const int r = threadIdx.x >> 2;
     const int ks = kc * kChunk + (threadIdx.x & 3);
@@ -1354,8 +1354,10 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
         return TDQ_ERR_CUDA;
 
     const unsigned pieces = (unsigned)((e.tiles_m + e.tiles_n) * p.n_chunks);
-    if (pow2_steps)
+    if (pow2_steps) {
+        if (cudaMemsetAsync(workspace, 0, 16, stream) != cudaSuccess) return TDQ_ERR_CUDA;
         expand_pow2_kernel<<<pieces, kExpandThreads, 0, stream>>>(e, act_group / 32, (int32_t)(I_pad / act_group));
+    }
     else if (i8)
         expand_kernel<true><<<pieces, kExpandThreads, 0, stream>>>(e);
     else
