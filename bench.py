@@ -57,7 +57,7 @@ def load_peaks():
 
 
 def workload(name):
-    return {"cfg2": si.config2, "cfg3": si.config3, "cfg4": si.config4}[name]()
+    return {"cfg1": si.config1, "cfg2": si.config2, "cfg3": si.config3, "cfg4": si.config4}[name]()
 
 
 def quant_bytes(M, C, esize, g=32):
@@ -292,6 +292,58 @@ def sweep_leg(tdq, dev):
                 graph_tops=2.0 * macs / (graph_ms * 1e-3) / 1e12, graph_gbs=(xbytes + ybytes) / (graph_ms * 1e-3) / 1e9)
 
 
+def small_configs_leg(tdq, dev, peaks):
+    """cfg1-cfg3 (launch-bound sizes): per call from a graph over rotating buffers, with both roofline fractions."""
+    import torch
+    out = {}
+    for name in ("cfg1", "cfg2", "cfg3"):
+        case = workload(name)
+        M, C, O = case.M, case.C, case.O
+        esz = 2 if case.x_is_bf16 else 4
+        xh = torch.from_numpy(case.x.reshape(M, C).view(np.int16).copy()).view(torch.bfloat16) if case.x_is_bf16 \
+            else torch.from_numpy(case.x.reshape(M, C).copy())
+        n = max(2, int(np.ceil(2.5 * L2_BYTES / (quant_bytes(M, C, esz) + M * O * 4))))
+        n = min(n, 48)
+        xs = [xh.to(dev) for _ in range(n)]
+        wc, ws = tdq.quantize_weight(torch.from_numpy(case.w).to(dev), 32)
+        codes = [torch.empty((M, C // 2), dtype=torch.uint8, device=dev) for _ in range(n)]
+        scales = [torch.empty((M, C // 32), dtype=torch.float32, device=dev) for _ in range(n)]
+        ys = [torch.empty((M, O), dtype=torch.float32, device=dev) for _ in range(n)]
+        wsp = tdq.linear_workspace(M, C, O, 32, dev)
+        p = tdq.default_act_params()
+        q_ms = time_graph(lambda i: tdq.quantize_act(xs[i % n], p, codes=codes[i % n], scale=scales[i % n]), 2 * n)
+        l_ms = time_graph(lambda i: tdq.w4a4_linear(codes[i % n], scales[i % n], wc, ws, y=ys[i % n], workspace=wsp), 2 * n)
+        f_ms = time_graph(lambda i: tdq.quant_linear_fused(xs[i % n], wc, ws, y=ys[i % n], workspace=wsp), 2 * n)
+        qb, lb, ops = quant_bytes(M, C, esz), linear_bytes(M, C, O), 2.0 * M * C * O
+        out[name] = dict(x=[int(v) for v in case.x.shape], O=O, buffer_sets=n,
+                         quantize_us=q_ms * 1e3, quantize_gbs=qb / (q_ms * 1e-3) / 1e9, quantize_frac_hbm=qb / (q_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                         linear_us=l_ms * 1e3, linear_tops=ops / (l_ms * 1e-3) / 1e12, linear_gbs=lb / (l_ms * 1e-3) / 1e9,
+                         linear_frac_hbm=lb / (l_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], linear_bound="hbm", fused_us=f_ms * 1e3)
+    return out
+
+
+def probe_leg(tdq, dev, peaks):
+    """A compute-bound shape (16384 x 4096 -> 4096, bf16 output) with per-32 groups and with one group per token."""
+    import torch
+    M = I = 16384
+    I = O = 4096
+    torch.manual_seed(1)
+    xc = torch.randint(0, 256, (M, I // 2), dtype=torch.uint8, device=dev)
+    wc = torch.randint(0, 256, (O, I // 2), dtype=torch.uint8, device=dev)
+    ws = torch.rand((O,), device=dev) + 0.5
+    ys = [torch.empty((M, O), dtype=torch.bfloat16, device=dev) for _ in range(2)]
+    out = {}
+    for g in (32, I):
+        xs = torch.rand((M, I // g), device=dev) + 0.5
+        wsp = tdq.linear_workspace(M, I, O, g, dev)
+        ms = time_graph(lambda i: tdq.w4a4_linear(xc, xs, wc, ws, g=g, y=ys[i % 2], workspace=wsp), 4, replays=3)
+        tops = 2.0 * M * I * O / (ms * 1e-3) / 1e12
+        out["g%d" % g] = dict(ms=ms, tops=tops, frac_int8=tops / (2.0 * peaks["bf16_tflops"]), frac_int8_4500=tops / 4500.0)
+    out["shape"] = [M, I, O]
+    out["y_dtype"] = "bf16"
+    return out
+
+
 def run_tdq(args):
     import torch
     import torch.distributed as dist
@@ -421,7 +473,7 @@ def run_tdq(args):
     e2e_ms = e0.elapsed_time(e1)
 
     total_ms, q_ms, l_ms, e2e_ms = max_over_ranks([total_ms, q_ms, l_ms, e2e_ms], dev, world)
-    fused = sweep = None
+    fused = sweep = small = probe = None
     q_iso_ms = l_iso_ms = None
     q_switch_ms = None
     q_nchw = None
@@ -467,6 +519,10 @@ def run_tdq(args):
         del xs, codes, scales, ys
         torch.cuda.empty_cache()
         sweep = sweep_leg(tdq, dev)
+        torch.cuda.empty_cache()
+        peaks_x = load_peaks()
+        small = small_configs_leg(tdq, dev, peaks_x)
+        probe = probe_leg(tdq, dev, peaks_x)
 
     if rank == 0:
         peaks = load_peaks()
@@ -512,7 +568,7 @@ def run_tdq(args):
                                cache="rotating %d buffer sets, %.0f MB per step (L2 is 126 MB)" % (nsets, step_bytes / 1e6),
                                launch=("CUDA graph of %d steps, replayed %d times" % (G, args.steps // G)) if G else "eager",
                                parallelism="rows sharded, %d replica(s)" % world),
-                   kernels=dict(quantize_act=q_kernel, quantize_act_nchw=q_nchw, w4a4_linear=l_kernel, w4a4_linear_pow2=pow2, fused=fused, sweep_cfg5=sweep,
+                   kernels=dict(quantize_act=q_kernel, quantize_act_nchw=q_nchw, w4a4_linear=l_kernel, w4a4_linear_pow2=pow2, fused=fused, sweep_cfg5=sweep, configs_1_to_3=small, compute_probe=probe,
                                 step_tokens_per_s=world * M * K / (total_ms * 1e-3)),
                    roofline=roof, clocks=clocks, gpu_launches=int(launches),
                    e2e=dict(value=e2e_value, unit="GB/s", ms_per_step=e2e_ms / e2e_steps,
@@ -536,7 +592,7 @@ def main():
     ap.add_argument("--steps", type=int, default=None, help="default: 1000 (10 for --impl reference)")
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="tdq", choices=["tdq", "reference"])
-    ap.add_argument("--workload", default="cfg4", choices=["cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--workload", default="cfg4", choices=["cfg1", "cfg2", "cfg3", "cfg4"])
     ap.add_argument("--cpu-rows", type=int, default=18464)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the fused-call and 32-layer sweep legs")
