@@ -127,7 +127,6 @@ struct LinArgs {
     const float* xscale;
     int32_t row_bytes;         // I_pad / 2
     int32_t unpack_a;
-    int32_t rotate_slots;      // fewer than four groups per tile, each of three steps or more: TMEM slots rotate across tiles
     // fused producer only: the activations themselves and the quantizer's parameters
     const void* x;
     int64_t x_stride;          // elements between rows of x
@@ -672,8 +671,6 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                 uint32_t q_a = 1, q_b = 1;     // parity to wait for on tempty of each slot; a fresh barrier passes parity 1
                 // otherwise: one slot at a time
                 uint32_t qm = 0xFu;            // the same parities as a mask, bit = slot
-                uint32_t slot = 0;             // restarts at 0 with every tile unless the slots rotate across tiles
-                bool slot_ready = false;       // the early answer about the next slot, if it was yes
                 for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
                     const int part = item % a.n_parts;
                     const int n_tiles = part_begin(part + 1) - part_begin(part);
@@ -681,10 +678,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                     const uint32_t ares_lo = desc_lo(ibuf_s + ib * a.ibuf_bytes + a_in_ibuf);
                     for (int tl = 0; tl < n_tiles && ok; ++tl) {
                         int sub = 0;
-                        if (!a.rotate_slots) {
-                            slot = 0;
-                            slot_ready = false;
-                        }
+                        uint32_t slot = 0;
+                        bool slot_ready = false;   // the early answer about the next slot, if it was yes
                         uint32_t a_lo = ares_lo;   // resident: walks through the item's A blocks
                         for (int k0 = 0; k0 < n_steps && ok; k0 += kChunk) {
                             ok = mbar_wait_warp(&c->full[s], ph, c, a.status, 4u);
@@ -1033,10 +1028,6 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
         uint32_t tfull_s = smem_u32(&c->tfull[0]), tempty_s = smem_u32(&c->tempty[0]), tmem_row_r = tmem_row;
         // opaque to the compiler: kept in registers instead of being recomputed from the thread index at every use
         asm volatile("" : "+r"(tfull_s), "+r"(tempty_s), "+r"(tmem_row_r));
-        const std::integral_constant<uint32_t, 0> u0{};
-        const std::integral_constant<uint32_t, 1> u1{};
-        const std::integral_constant<uint32_t, 2> u2{};
-        const std::integral_constant<uint32_t, 3> u3{};
         auto request = [&](auto u_tag, bool ready) {
             constexpr uint32_t U = decltype(u_tag)::value;
             if (!__all_sync(0xffffffffu, ready)) ok = mbar_wait_warp(&c->tfull[U], p_full[U], c, a.status, 2u);
@@ -1044,15 +1035,6 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
             tc_fence_after();
             if (FUSED) tmem_ld16(tmem_row_r + U * kBN, v);
             else tmem_ld32(tmem_row_r + U * kBN, v);
-        };
-        uint32_t cur_slot = 0;      // rotating slots: the slot of the group that is next to be consumed
-        auto request_rt = [&](bool ready) {
-            switch (cur_slot) {
-                case 0: request(u0, ready); break;
-                case 1: request(u1, ready); break;
-                case 2: request(u2, ready); break;
-                default: request(u3, ready); break;
-            }
         };
         auto consume = [&](auto u_tag, uint32_t scale_q, int k) -> bool {
             constexpr uint32_t U = decltype(u_tag)::value, N = (U + 1) & (kSlots - 1);
@@ -1081,6 +1063,11 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
             for (int q = 0; q < kLand / 2; ++q) fma2(yacc[(FUSED ? kLand / 2 : 0) + q], pack2(v[2 * q], v[2 * q + 1]), d2);
             return next_ready;
         };
+        const std::integral_constant<uint32_t, 0> u0{};
+        const std::integral_constant<uint32_t, 1> u1{};
+        const std::integral_constant<uint32_t, 2> u2{};
+        const std::integral_constant<uint32_t, 3> u3{};
+
         if (item < n_items) {
             begin_item();
             if (ok) {
@@ -1091,28 +1078,6 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
             while (ok && item < n_items) {
                 // one tile; the load of its first group is in flight
                 const int Kg = a.Kg;
-                if (a.rotate_slots) {
-                    // Fewer than four groups per tile: the slots rotate across tiles, so that the tensor core can
-                    // run up to four groups ahead of the epilogues instead of one tile.
-#pragma unroll 1
-                    for (int k = 0; k < Kg && ok; ++k) {
-                        const uint32_t sq = my_scale_s + (uint32_t)k * kScaleBlock - cur_slot * kScaleBlock;
-                        const int kd = k - (int)cur_slot;
-                        bool r;
-                        switch (cur_slot) {
-                            case 0: r = consume(u0, sq, kd); break;
-                            case 1: r = consume(u1, sq, kd); break;
-                            case 2: r = consume(u2, sq, kd); break;
-                            default: r = consume(u3, sq, kd); break;
-                        }
-                        cur_slot = (cur_slot + 1) & (kSlots - 1);
-                        if (k + 1 < Kg) request_rt(r);
-                    }
-                    if (!ok) break;
-                    finish_tile();
-                    if (ok && item < n_items) request_rt(false);
-                    continue;
-                }
                 uint32_t scale_q = my_scale_s;
                 int k = 0;
 #pragma unroll 1
@@ -1370,7 +1335,6 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
     a.half_strips = half_strips ? 1 : 0;
     a.out_scale = i8 ? 0.00390625f : 262144.0f;
     a.xcodes = xcodes; a.xscale = xscale; a.row_bytes = e.row_bytes; a.unpack_a = unpack_a ? 1 : 0;
-    a.rotate_slots = (a.Kg < 4 && a.steps_per_grp >= 3) ? 1 : 0;
     a.x = fx ? fx->x : nullptr;
     a.x_stride = fx ? fx->row_stride : 0;
     a.seven_tau = fx ? fx->seven_tau : 0.0f;
