@@ -399,19 +399,21 @@ def run_tdq(args):
         raise RuntimeError("linear kernel reported a device-side timeout: 0x%x" % detail)
 
     # The timed steps are replayed from a CUDA graph, so that the kernels run back to back and the
-    # device-side events between them measure kernels, not the host's launch path.  A graph holds
-    # G steps (a multiple of the buffer rotation, each with its own three events) and is replayed
-    # K / G times; per-kernel times come from the events of the last replay, the step time from
-    # the events around all replays.
+    # events measure kernels, not the host's launch path.  A graph holds G steps (a multiple of the
+    # buffer rotation) and is replayed K / G times between two events: the step time.  The graph has
+    # no event nodes inside: an event record between two kernel nodes costs about 7 us on this
+    # hardware (cfg4: 157.8 us per step with two of them per step, 143.8 us without), which is
+    # measurement, not the path.  Each kernel's own duration is timed the same way right after, from a
+    # graph of that call alone over rotating buffers (inputs beyond 2.5 x L2), events around its launches.
     G = graph_steps(args.steps, nsets) if not args.eager else 0
     sampler = ClockSampler(local)
     launches0 = tdq.kernel_launch_count()
     if G:
-        evs = [[torch.cuda.Event(enable_timing=True, external=True) for _ in range(3)] for _ in range(G)]
+        evs = None
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph):
             for i in range(G):
-                step(args.warmup + i, evs[i])
+                step(args.warmup + i)
         launches_per_replay = tdq.kernel_launch_count() - launches0
         graph.replay()                       # untimed: uploads the graph
         barrier()
@@ -441,9 +443,20 @@ def run_tdq(args):
         launches = tdq.kernel_launch_count() - launches0
     clocks = sampler.stop() if rank == 0 else None
     total_ms = t_begin.elapsed_time(t_end)
-    n_ev = len(evs)
-    q_ms = sum(e[0].elapsed_time(e[1]) for e in evs) * args.steps / n_ev
-    l_ms = sum(e[1].elapsed_time(e[2]) for e in evs) * args.steps / n_ev
+    n_iso = min(64, max(nsets, int(np.ceil(2.5 * L2_BYTES / (M * C * esize)))))   # input sets of the quantizer alone
+    if G:
+        xi = xs + [xs[0].clone() for _ in range(n_iso - nsets)]
+        n_q = n_iso * max(1, min(args.steps, 64) // n_iso)
+        q_call_ms = time_graph(lambda i: tdq.quantize_act(xi[i % n_iso], params, codes=codes[i % nsets], scale=scales[i % nsets]),
+                               n_q, replays=max(1, args.steps // n_q))
+        l_call_ms = time_graph(lambda i: tdq.w4a4_linear(codes[i % nsets], scales[i % nsets], wcodes, wscale, y=ys[i % nsets],
+                                                         workspace=wsp), G, replays=args.steps // G)
+        q_ms, l_ms = q_call_ms * args.steps, l_call_ms * args.steps
+        barrier()
+    else:
+        n_ev = len(evs)
+        q_ms = sum(e[0].elapsed_time(e[1]) for e in evs) * args.steps / n_ev
+        l_ms = sum(e[1].elapsed_time(e[2]) for e in evs) * args.steps / n_ev
 
     # end to end: pinned host X in, host Y out, through the host-buffer entry point
     xh = x_host.pin_memory()
@@ -481,10 +494,21 @@ def run_tdq(args):
     if world == 1 and not args.no_extras:
         # each kernel on its own, launched back to back from a graph over rotating buffers: no other
         # kernel and no event node between two launches (the in-step figures above include those gaps)
-        n_iso = max(nsets, int(np.ceil(2.5 * L2_BYTES / (M * C * esize))))
-        xi = xs + [xs[0].clone() for _ in range(n_iso - nsets)]
-        q_iso_ms = time_graph(lambda i: tdq.quantize_act(xi[i % n_iso], params, codes=codes[i % nsets], scale=scales[i % nsets]),
-                              4 * n_iso)
+        if not G:
+            xi = xs + [xs[0].clone() for _ in range(n_iso - nsets)]
+        # the same steps with an event record in front of and behind every call (what a graph with event
+        # nodes measures; kept to show the difference)
+        evx = [[torch.cuda.Event(enable_timing=True, external=True) for _ in range(3)] for _ in range(2 * nsets)]
+        gx = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gx):
+            for i in range(2 * nsets):
+                step(i, evx[i])
+        gx.replay()
+        gx.replay()
+        torch.cuda.synchronize()
+        q_iso_ms = sum(e[0].elapsed_time(e[1]) for e in evx) / len(evx)
+        l_iso_ms = sum(e[1].elapsed_time(e[2]) for e in evx) / len(evx)
+        del gx
         # the quantizer with one or both bounds switched off (the paper's C1-only, C2-only and
         # DSTG-only ablation settings), back to back like the line above
         q_switch_ms = {}
@@ -506,8 +530,6 @@ def run_tdq(args):
         q_nchw = dict(name="tdq_quantize_act_nchw", x=[32, C, 24, 24], ms=q_nchw_ms,
                       gbs=quant_bytes(Mf, C, esize) / (q_nchw_ms * 1e-3) / 1e9)
         del fm, fcodes, fscale
-        l_iso_ms = time_graph(lambda i: tdq.w4a4_linear(codes[i % nsets], scales[i % nsets], wcodes, wscale, y=ys[i % nsets],
-                                                        workspace=wsp), 8 * nsets)
         # the power-of-two step variant (not the paper's quantizer): its quantizer and its linear layer
         p2 = tdq.act_params(flags=tdq.ENABLE_C1 | tdq.ENABLE_C2 | tdq.POW2_STEP)
         tdq.quantize_act(xs[0], p2, codes=codes[0], scale=scales[0])
@@ -535,17 +557,18 @@ def run_tdq(args):
         int8_peak = 2.0 * peaks["bf16_tflops"]            # nominal int8 : bf16 ratio on the measured bf16 peak
         q_kernel = dict(name="tdq_quantize_act", ms=q_ms / K, gbs=q_gbs, frac_hbm=q_gbs / peaks["hbm_gbs"],
                         frac_hbm_8tbs=q_gbs / 8000.0, algorithmic_bytes=qb)
+        timing = ("events around launches of this call alone, replayed from a CUDA graph over rotating buffers" if G
+                  else "events around every call, launched from the host")
+        q_kernel["timing"] = timing
         if q_iso_ms:
-            q_kernel.update(back_to_back_ms=q_iso_ms, back_to_back_gbs=qb / (q_iso_ms * 1e-3) / 1e9,
-                            back_to_back_frac_hbm=qb / (q_iso_ms * 1e-3) / 1e9 / peaks["hbm_gbs"])
-            q_kernel["back_to_back_ms_by_setting"] = q_switch_ms
+            q_kernel.update(ms_between_event_nodes_in_step=q_iso_ms, ms_by_setting=q_switch_ms)
         l_kernel = dict(name="tdq_w4a4_linear", ms=l_ms / K, tops=l_tops, frac_int8=l_tops / int8_peak,
                         frac_int8_4500=l_tops / 4500.0, gbs=l_gbs, frac_hbm=l_gbs / peaks["hbm_gbs"],
                         algorithmic_bytes=lb, ops=ops,
                         bound="hbm" if lb / peaks["hbm_gbs"] / 1e9 > ops / int8_peak / 1e12 else "tensor")
+        l_kernel["timing"] = timing
         if l_iso_ms:
-            l_kernel.update(back_to_back_ms=l_iso_ms, back_to_back_tops=ops / (l_iso_ms * 1e-3) / 1e12,
-                            back_to_back_gbs=lb / (l_iso_ms * 1e-3) / 1e9)
+            l_kernel.update(ms_between_event_nodes_in_step=l_iso_ms)
         if l_ms >= q_ms:
             if l_kernel["bound"] == "hbm":
                 roof = dict(kernel="tdq_w4a4_linear", bound="hbm", achieved=l_gbs, peak=peaks["hbm_gbs"],
@@ -566,7 +589,7 @@ def run_tdq(args):
                    config=dict(workload=case.name, x=[int(v) for v in case.x.shape], w=[int(v) for v in case.w.shape],
                                g=32, tau=1.0, zr=0.2, y_dtype="f32",
                                cache="rotating %d buffer sets, %.0f MB per step (L2 is 126 MB)" % (nsets, step_bytes / 1e6),
-                               launch=("CUDA graph of %d steps, replayed %d times" % (G, args.steps // G)) if G else "eager",
+                               launch=("CUDA graph of %d steps without event nodes, replayed %d times; each kernel timed from a graph of its call alone" % (G, args.steps // G)) if G else "eager",
                                parallelism="rows sharded, %d replica(s)" % world),
                    kernels=dict(quantize_act=q_kernel, quantize_act_nchw=q_nchw, w4a4_linear=l_kernel, w4a4_linear_pow2=pow2, fused=fused, sweep_cfg5=sweep, configs_1_to_3=small, compute_probe=probe,
                                 step_tokens_per_s=world * M * K / (total_ms * 1e-3)),
