@@ -512,3 +512,52 @@ def test_fused_and_power_of_two_random_shapes(tdq, M, C, O, g, bf16_out, with_bi
     # power-of-two steps at the drawn group size against the exact layer's oracle
     y, ref, _ = _pow2_case(tdq, x, False, w, g=g, bias=bias, out_dtype=dt)
     compare_y(y, ref, C, out_eps=2.0 ** -8 if bf16_out else 0.0)
+
+
+# ------------------------------------------------------------------------------------------
+# the launch configuration the benchmark times: steps replayed from a CUDA graph over rotating buffers
+
+def test_full_size_step_replayed_from_a_graph_matches_oracle_on_sampled_rows(tdq):
+    case = si.config(4)
+    x = case.x.reshape(-1, case.C)
+    M, C, O = x.shape[0], case.C, case.w.shape[0]
+    nsets = 2
+    xt = to_cuda(x, bf16=case.x_is_bf16)
+    wc, ws = tdq.quantize_weight(to_cuda(case.w))
+    codes = [torch.zeros((M, C // 2), dtype=torch.uint8, device="cuda") for _ in range(nsets)]
+    scales = [torch.zeros((M, C // 32), dtype=torch.float32, device="cuda") for _ in range(nsets)]
+    ys = [torch.zeros((M, O), dtype=torch.float32, device="cuda") for _ in range(nsets)]
+    wsp = tdq.linear_workspace(M, C, O, 32, "cuda")
+    params = tdq.default_act_params()
+
+    def step(i):
+        s = i % nsets
+        tdq.quantize_act(xt, params, codes=codes[s], scale=scales[s])
+        tdq.w4a4_linear(codes[s], scales[s], wc, ws, y=ys[s], workspace=wsp)
+
+    step(0)
+    torch.cuda.synchronize()
+    y_eager = ys[0].clone()
+    for t in codes + scales + ys:
+        t.zero_()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for i in range(2 * nsets):
+            step(i)
+    for t in codes + scales + ys:
+        t.zero_()
+    graph.replay()
+    graph.replay()
+    torch.cuda.synchronize()
+    st, detail = tdq.workspace_status(wsp)
+    assert st == tdq.OK, "device wait ran out: 0x%x" % detail
+    for s in range(nsets):
+        assert torch.equal(ys[s].view(torch.int32), y_eager.view(torch.int32))      # every set, same bits as the eager call
+    rng = np.random.default_rng(44)
+    rows = np.unique(np.concatenate([rng.choice(M, 96, replace=False), [0, 127, 128, M - 1]]))
+    xa = oracle.quantize_act(x[rows])
+    wq = oracle.quantize_weight(case.w)
+    ref = oracle.w4a4_linear(xa["codes"], xa["scale"], wq["codes"], wq["scale"])
+    np.testing.assert_array_equal(codes[1].cpu().numpy()[rows], xa["codes"])
+    np.testing.assert_array_equal(scales[1].cpu().numpy()[rows], xa["scale"])
+    compare_y(ys[1].cpu().numpy()[rows], ref, C // 32)
