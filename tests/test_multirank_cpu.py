@@ -56,3 +56,31 @@ def test_graph_steps_divides_the_step_count_and_respects_the_buffer_rotation():
         assert K % G == 0 and 1 <= G <= max(K, 64)
         # either a whole number of rotations per graph, or one graph that holds every step
         assert G % nsets == 0 or G == K
+
+
+def _run_reference_arm(extra_env):
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ)
+    env.update(extra_env)
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--impl", "reference", "--steps", "1", "--warmup", "1",
+                        "--workload", "cfg1"], capture_output=True, text=True, env=env, cwd=root, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
+    return [json.loads(l) for l in lines]
+
+
+def test_reference_arm_prints_the_contract_line_on_the_host_cores():
+    (line,) = _run_reference_arm({"RANK": "0", "WORLD_SIZE": "1"})
+    assert line["impl"] == "reference" and line["unit"] == "GB/s" and line["value"] > 0 and line["higher_is_better"] is True
+    assert line["steps"] == 1 and line["warmup"] == 1 and line["ms_per_step"] > 0 and line["gpu_launches"] == 0
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] >= 1
+    assert line["cpu_baseline"]["value"] == line["value"] and line["cpu_baseline"]["sample"]
+    assert line["e2e"] == dict(value=line["value"], unit="GB/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0)
+    assert line["config"]["workload"].startswith("cfg1")
+
+
+def test_reference_arm_is_silent_on_other_ranks():
+    assert _run_reference_arm({"RANK": "1", "WORLD_SIZE": "2", "LOCAL_RANK": "1"}) == []
