@@ -516,6 +516,9 @@ def run_tdq(args):
             pf = tdq.act_params(flags=flags)
             q_switch_ms[label] = time_graph(lambda i: tdq.quantize_act(xi[i % n_iso], pf, codes=codes[i % nsets],
                                                                        scale=scales[i % nsets]), 4 * n_iso)
+        pp = tdq.act_params(p=0.95)     # base radius = 31st of the 32 magnitudes (Supp. S4.8's percentile option)
+        q_switch_ms["percentile_0.95"] = time_graph(lambda i: tdq.quantize_act(xi[i % n_iso], pp, codes=codes[i % nsets],
+                                                                               scale=scales[i % nsets]), 4 * n_iso)
         # the fixed-radius control: no reductions, the speed limit of a one-pass quantizer of this size
         q_switch_ms["fixed_radius"] = time_graph(lambda i: tdq.quantize_act_fixed(xi[i % n_iso], 1.0, 32, codes=codes[i % nsets],
                                                                                  scale=scales[i % nsets]), 4 * n_iso)

@@ -112,10 +112,35 @@ __device__ __forceinline__ uint32_t nibble_ieee(float x, float c, float delta) {
     return (uint32_t)quantize_ieee(x, c, delta) & 0xFu;
 }
 
+// K-th smallest of 32 magnitudes given as two sorted halves (even and odd channels of a bf16 group in
+// the low and high 16 bits of s[0..15]; s[0..15] and s[16..31] of an fp32 group): the maximum over
+// i + j = K - 1 of min(E[i], O[j]), an index past the end counting as +inf.
+template <int K>
+__device__ __forceinline__ uint32_t kth_of_sorted_halves_u16(const uint32_t (&s)[16]) {
+    constexpr int lo_i = (K > 16) ? K - 16 : 0;
+    constexpr int hi_i = (K - 1 < 15) ? K - 1 : 15;
+    constexpr int mid_i = (lo_i + hi_i) / 2;
+    uint32_t r = (K > 16) ? s[(K > 16) ? K - 17 : 0] : 0u;
+#pragma unroll
+    for (int i = lo_i; i <= mid_i && i <= hi_i; ++i)
+        r = __vmaxu2(r, __vminu2(s[i], __byte_perm(s[K - 1 - i], 0u, 0x1032u)));
+    return max(r & 0xffffu, r >> 16);
+}
+template <int K>
+__device__ __forceinline__ float kth_of_sorted_halves_f32(const float (&s)[32]) {
+    constexpr int lo_i = (K > 16) ? K - 16 : 0;
+    constexpr int hi_i = (K - 1 < 15) ? K - 1 : 15;
+    float r = (K > 16) ? fmaxf(s[(K > 16) ? K - 17 : 0], s[(K > 16) ? K - 1 : 16]) : 0.0f;
+#pragma unroll
+    for (int i = lo_i; i <= hi_i; ++i) r = fmaxf(r, fminf(s[i], s[16 + K - 1 - i]));
+    return r;
+}
+
 // One group held in registers (w: 16 packed bf16 pairs or 32 floats, in channel order): statistics,
 // projection, quantization.  out: the group's 32 two's complement nibbles, channel 8 w + n in
-// nibble n of word w; delta: its step.
-template <bool BF16, int KZR>
+// nibble n of word w; delta: its step.  KB: rank of the base radius among the magnitudes (32: the maximum,
+// Eq. 5; less: the percentile option of Supp. S4.8, which takes the group's KB-th smallest magnitude).
+template <bool BF16, int KZR, int KB = 32>
 __device__ __forceinline__ void quantize_group32(const uint32_t (&w)[BF16 ? 16 : 32], float seven_tau, uint32_t flags,
                                                  uint32_t (&out)[4], float& delta) {
     auto get = [&](int i) -> float {
@@ -125,7 +150,31 @@ __device__ __forceinline__ void quantize_group32(const uint32_t (&w)[BF16 ? 16 :
 
     // base radius, rank-KZR magnitude, moments
     float c_base, thr = 0.0f;
-    if (BF16) {
+    if (KB < 32) {
+        // percentile base radius: both ranks come from the same two sorted halves
+        if (BF16) {
+            uint32_t s[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) s[i] = w[i] & 0x7fff7fffu;
+#define TDQ_CE(i, j) { uint32_t lo_ = __vminu2(s[i], s[j]); s[j] = __vmaxu2(s[i], s[j]); s[i] = lo_; }
+#include "sort16_network.inc"
+#undef TDQ_CE
+            c_base = __uint_as_float(kth_of_sorted_halves_u16<KB>(s) << 16);
+            if (flags & TDQ_ENABLE_C2) thr = __uint_as_float(kth_of_sorted_halves_u16<KZR>(s) << 16);
+        } else {
+            float s[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) s[i] = fabsf(__uint_as_float(w[i]));
+#define TDQ_CE(i, j) { float lo_ = fminf(s[i], s[j]); s[j] = fmaxf(s[i], s[j]); s[i] = lo_; }
+#include "sort16_network.inc"
+#undef TDQ_CE
+#define TDQ_CE(i, j) { float lo_ = fminf(s[16 + i], s[16 + j]); s[16 + j] = fmaxf(s[16 + i], s[16 + j]); s[16 + i] = lo_; }
+#include "sort16_network.inc"
+#undef TDQ_CE
+            c_base = kth_of_sorted_halves_f32<KB>(s);
+            if (flags & TDQ_ENABLE_C2) thr = kth_of_sorted_halves_f32<KZR>(s);
+        }
+    } else if (BF16) {
         // |x| of a bf16 is a 15-bit key whose unsigned order is the numeric order, so the network
         // runs on packed 16-bit integer min/max (two channels per instruction, integer pipe)
         uint32_t s[16];

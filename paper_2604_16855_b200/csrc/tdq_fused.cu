@@ -19,6 +19,7 @@ extern "C" tdq_status tdq_quant_linear_fused(const void* x, tdq_dtype x_dtype, i
     if (p->group_size != 32 || C % 32 != 0 || !act_fast_path_ok(x, x_dtype, C, row_stride_elems, p))
         return TDQ_ERR_UNSUPPORTED;
     if ((p->flags & TDQ_ENABLE_C2) && rank_of(p->zr, 32) != 7) return TDQ_ERR_UNSUPPORTED;
+    if (rank_of(p->base_percentile, 32) != 32) return TDQ_ERR_UNSUPPORTED;   // the producer takes the maximum as base radius
     FusedSrc fx;
     fx.x = x;
     fx.row_stride = row_stride_elems;

@@ -135,17 +135,17 @@ __global__ void __launch_bounds__(kGenericWarps * 32) act_generic_kernel(ActArgs
 constexpr int kFastThreads = 256;   // groups per CTA tile
 
 // One group: quantize it in registers, write its 16 code bytes and its scale.
-template <bool BF16, int KZR>
+template <bool BF16, int KZR, int KB = 32>
 __device__ __forceinline__ void process_group(const uint32_t (&w)[BF16 ? 16 : 32], const ActArgs& a, int64_t gi) {
     uint32_t out[4];
     float delta;
-    quantize_group32<BF16, KZR>(w, a.seven_tau, a.flags, out, delta);
+    quantize_group32<BF16, KZR, KB>(w, a.seven_tau, a.flags, out, delta);
     reinterpret_cast<uint4*>(a.codes)[gi] = make_uint4(out[0], out[1], out[2], out[3]);
     a.scale[gi] = delta;
     if (a.offset) a.offset[gi] = 0.0f;
 }
 
-template <bool BF16, int KZR>
+template <bool BF16, int KZR, int KB = 32>
 __global__ void __launch_bounds__(kFastThreads) act_g32_kernel(ActArgs a) {
     constexpr int kGroupBytes = BF16 ? 64 : 128;
     constexpr int kChunks = kGroupBytes / 16;          // 16-byte chunks per group
@@ -194,7 +194,7 @@ __global__ void __launch_bounds__(kFastThreads) act_g32_kernel(ActArgs a) {
             w[4 * p + 0] = v.x; w[4 * p + 1] = v.y; w[4 * p + 2] = v.z; w[4 * p + 3] = v.w;
         }
     }
-    process_group<BF16, KZR>(w, a, gi);
+    process_group<BF16, KZR, KB>(w, a, gi);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -239,7 +239,7 @@ __device__ __forceinline__ bool ring_wait(uint64_t* bar, uint32_t parity, volati
     return true;
 }
 
-template <bool BF16, int KZR>
+template <bool BF16, int KZR, int KB = 32>
 __global__ void __launch_bounds__(kRingThreads) act_g32_ring_kernel(ActArgs a, int64_t n_tiles) {
     constexpr int kGroupBytes = BF16 ? 64 : 128;
     constexpr int kChunks = kGroupBytes / 16;
@@ -298,11 +298,11 @@ __global__ void __launch_bounds__(kRingThreads) act_g32_ring_kernel(ActArgs a, i
         if ((t & 31) == 0)
             asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(ring_smem_u32(&empty[s])) : "memory");
         if (++s == kStages) { s = 0; ph ^= 1; }
-        if (gi < a.total_groups) process_group<BF16, KZR>(w, a, gi);
+        if (gi < a.total_groups) process_group<BF16, KZR, KB>(w, a, gi);
     }
 }
 
-template <bool BF16, int KZR>
+template <bool BF16, int KZR, int KB = 32>
 cudaError_t launch_ring(const ActArgs& a, cudaStream_t st) {
     constexpr int kStages = BF16 ? kRingStagesBf16 : kRingStagesF32;
     constexpr int smem = kStages * kFastThreads * (BF16 ? 64 : 128);
@@ -314,13 +314,13 @@ cudaError_t launch_ring(const ActArgs& a, cudaStream_t st) {
         if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return cudaErrorUnknown;
     }
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(act_g32_ring_kernel<BF16, KZR>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        cudaError_t e = cudaFuncSetAttribute(act_g32_ring_kernel<BF16, KZR, KB>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
     const int64_t n_tiles = (a.total_groups + kFastThreads - 1) / kFastThreads;
     const int64_t grid = n_tiles < 2 * n_sm ? n_tiles : 2 * n_sm;
-    act_g32_ring_kernel<BF16, KZR><<<(unsigned)grid, kRingThreads, smem, st>>>(a, n_tiles);
+    act_g32_ring_kernel<BF16, KZR, KB><<<(unsigned)grid, kRingThreads, smem, st>>>(a, n_tiles);
     return cudaGetLastError();
 }
 
@@ -328,6 +328,19 @@ template <bool BF16>
 cudaError_t launch_fast(const ActArgs& a, cudaStream_t st) {
     const int64_t blocks = (a.total_groups + kFastThreads - 1) / kFastThreads;
     dim3 grid((unsigned)blocks), block(kFastThreads);
+    if (a.k_base != 32) {        // percentile base radius: ranks 29..31 beside the default zero-bin rank
+        if (a.k_zr != 7) return cudaErrorInvalidValue;
+        switch (a.k_base) {
+#define TDQ_CASE(KB_)                                                                  \
+            case KB_:                                                                  \
+                if (a.row_stride == a.C) return launch_ring<BF16, 7, KB_>(a, st);      \
+                act_g32_kernel<BF16, 7, KB_><<<grid, block, 0, st>>>(a);               \
+                return cudaGetLastError();
+            TDQ_CASE(29) TDQ_CASE(30) TDQ_CASE(31)
+#undef TDQ_CASE
+            default: return cudaErrorInvalidValue;
+        }
+    }
     if (a.row_stride == a.C) {   // dense rows: the persistent ring kernel
         switch (a.k_zr) {
 #define TDQ_CASE(KZ) case KZ: return launch_ring<BF16, KZ>(a, st);
@@ -489,6 +502,12 @@ __global__ void __launch_bounds__(256) act_fixed_kernel(FixedArgs f) {
 }
 
 bool fast_rank(int k) { return k == 4 || k == 7 || k == 10 || k == 13 || k == 16 || k == 32; }
+// base radius: the maximum, or one of the three ranks below it together with the default zero-bin rank
+bool fast_base_rank(const tdq_act_params* p) {
+    const int kb = rank_of(p->base_percentile, 32);
+    if (kb == 32) return true;
+    return kb >= 29 && (!(p->flags & TDQ_ENABLE_C2) || rank_of(p->zr, 32) == 7);
+}
 
 }  // namespace
 
@@ -509,7 +528,7 @@ bool act_fast_path_ok(const void* x, tdq_dtype dt, int64_t C, int64_t stride, co
     const int32_t g = p->group_size;
     const int64_t esize = dt == TDQ_BF16 ? 2 : 4;
     return g == 32 && C % 32 == 0 && (reinterpret_cast<uintptr_t>(x) % 16 == 0) &&
-           (stride * esize) % 16 == 0 && rank_of(p->base_percentile, g) == g &&
+           (stride * esize) % 16 == 0 && fast_base_rank(p) &&
            (!(p->flags & TDQ_ENABLE_C2) || fast_rank(rank_of(p->zr, g)));
 }
 

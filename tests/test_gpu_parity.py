@@ -80,6 +80,25 @@ def test_quantizer_percentile_and_odd_rank_take_generic_kernel(tdq):
         compare_quantizer(x, 32, ref, codes, scale)
 
 
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("p,flags", [(0.9, 3), (0.92, 3), (0.95, 3), (0.9, 1), (0.95, 0), (0.92, 2)])
+def test_quantizer_percentile_base_radius_on_the_fast_path(tdq, bf16, p, flags):
+    # ranks 29, 30 and 31 of 32 (Supp. S4.8's percentile option) on dense rows and on rows with a pitch
+    xs = [si.dc_offset_tokens(M=700, C=96), si.config1().x.reshape(-1, 64), si.edge_rows(C=64)]
+    for x in xs:
+        if bf16:
+            x = si.f32_to_bf16_bits(x)
+        ref, codes, scale = _quant_both(tdq, x, bf16, p=p, flags=flags)
+        rep = compare_quantizer(_f32(x, bf16), 32, ref, codes, scale)
+        assert rep["scale_exact_frac"] == 1.0, rep
+        wide = np.zeros((x.shape[0], x.shape[1] + 32), x.dtype)
+        wide[:, : x.shape[1]] = x
+        xt = to_cuda(wide, bf16=bf16)[:, : x.shape[1]]
+        c2, s2 = tdq.quantize_act(xt, tdq.act_params(p=p, flags=flags))
+        np.testing.assert_array_equal(c2.cpu().numpy(), codes)
+        np.testing.assert_array_equal(s2.cpu().numpy(), scale)
+
+
 def test_quantizer_row_stride_offset_output_and_empty(tdq):
     case = si.config2()
     bits = case.x.reshape(-1, 64)[:1000]
@@ -275,6 +294,9 @@ def test_fused_settings_and_refusals(tdq):
     assert e.value.code == tdq.ERR_UNSUPPORTED
     with pytest.raises(tdq.TdqError) as e:
         tdq.quant_linear_fused(xt, wc, ws, params=tdq.act_params(g=64))
+    assert e.value.code == tdq.ERR_UNSUPPORTED
+    with pytest.raises(tdq.TdqError) as e:          # a percentile base radius: the two-call path has it
+        tdq.quant_linear_fused(xt, wc, ws, params=tdq.act_params(p=0.95))
     assert e.value.code == tdq.ERR_UNSUPPORTED
     wide = torch.zeros((64, 2048), dtype=torch.bfloat16, device="cuda")
     wcw, wsw = tdq.quantize_weight(torch.zeros((32, 2048), device="cuda"))
