@@ -74,10 +74,10 @@ void tdq_default_act_params(tdq_act_params* p /* HOST, out */);
  *
  *   x          [B*N rows, C] row-major, x_dtype, consecutive rows row_stride_elems apart
  *              (>= C).  No alignment is required; 16-byte aligned x with C % 32 == 0,
- *              row_stride_elems % 8 == 0 and g == 32 takes the fast kernel (for the zero-bin
- *              ranks 4, 7, 10, 13, 16 and 32 with the maximum as base radius, and for base
- *              ranks 29-31 with zero-bin rank 7 or TDQ_ENABLE_C2 off; anything else takes a
- *              slower general kernel with the same results).
+ *              row_stride_elems % 8 == 0 and g == 32 takes the fast kernel (any zero-bin rank
+ *              with the maximum as base radius; base ranks 29-31 with zero-bin rank 7 or
+ *              TDQ_ENABLE_C2 off; anything else takes a much slower general kernel with the
+ *              same results).
  *   codes      [B*N, C_pad/2] bytes; byte j of a row holds channel 2j in its low nibble
  *              and channel 2j+1 in its high nibble, two's complement.
  *   scale      [B*N, K] float32, Delta_k.

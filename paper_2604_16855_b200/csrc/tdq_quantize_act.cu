@@ -324,6 +324,12 @@ cudaError_t launch_ring(const ActArgs& a, cudaStream_t st) {
     return cudaGetLastError();
 }
 
+// every zero-bin rank of a group of 32 has its instance of the two row-major kernels
+#define TDQ_ALL_RANKS \
+    TDQ_CASE(1) TDQ_CASE(2) TDQ_CASE(3) TDQ_CASE(4) TDQ_CASE(5) TDQ_CASE(6) TDQ_CASE(7) TDQ_CASE(8) \
+    TDQ_CASE(9) TDQ_CASE(10) TDQ_CASE(11) TDQ_CASE(12) TDQ_CASE(13) TDQ_CASE(14) TDQ_CASE(15) TDQ_CASE(16) \
+    TDQ_CASE(17) TDQ_CASE(18) TDQ_CASE(19) TDQ_CASE(20) TDQ_CASE(21) TDQ_CASE(22) TDQ_CASE(23) TDQ_CASE(24) \
+    TDQ_CASE(25) TDQ_CASE(26) TDQ_CASE(27) TDQ_CASE(28) TDQ_CASE(29) TDQ_CASE(30) TDQ_CASE(31) TDQ_CASE(32)
 template <bool BF16>
 cudaError_t launch_fast(const ActArgs& a, cudaStream_t st) {
     const int64_t blocks = (a.total_groups + kFastThreads - 1) / kFastThreads;
@@ -344,14 +350,14 @@ cudaError_t launch_fast(const ActArgs& a, cudaStream_t st) {
     if (a.row_stride == a.C) {   // dense rows: the persistent ring kernel
         switch (a.k_zr) {
 #define TDQ_CASE(KZ) case KZ: return launch_ring<BF16, KZ>(a, st);
-            TDQ_CASE(4) TDQ_CASE(7) TDQ_CASE(10) TDQ_CASE(13) TDQ_CASE(16) TDQ_CASE(32)
+            TDQ_ALL_RANKS
 #undef TDQ_CASE
             default: return cudaErrorInvalidValue;
         }
     }
     switch (a.k_zr) {
 #define TDQ_CASE(KZ) case KZ: act_g32_kernel<BF16, KZ><<<grid, block, 0, st>>>(a); break;
-        TDQ_CASE(4) TDQ_CASE(7) TDQ_CASE(10) TDQ_CASE(13) TDQ_CASE(16) TDQ_CASE(32)
+        TDQ_ALL_RANKS
 #undef TDQ_CASE
         default: return cudaErrorInvalidValue;
     }
@@ -501,6 +507,7 @@ __global__ void __launch_bounds__(256) act_fixed_kernel(FixedArgs f) {
     }
 }
 
+// the zero-bin ranks the channel-major kernel is instantiated for (those of the paper's sweep over zr)
 bool fast_rank(int k) { return k == 4 || k == 7 || k == 10 || k == 13 || k == 16 || k == 32; }
 // base radius: the maximum, or one of the three ranks below it together with the default zero-bin rank
 bool fast_base_rank(const tdq_act_params* p) {
@@ -528,8 +535,7 @@ bool act_fast_path_ok(const void* x, tdq_dtype dt, int64_t C, int64_t stride, co
     const int32_t g = p->group_size;
     const int64_t esize = dt == TDQ_BF16 ? 2 : 4;
     return g == 32 && C % 32 == 0 && (reinterpret_cast<uintptr_t>(x) % 16 == 0) &&
-           (stride * esize) % 16 == 0 && fast_base_rank(p) &&
-           (!(p->flags & TDQ_ENABLE_C2) || fast_rank(rank_of(p->zr, g)));
+           (stride * esize) % 16 == 0 && fast_base_rank(p);   // every zero-bin rank has its instance
 }
 
 }  // namespace tdq

@@ -73,7 +73,21 @@ def test_quantizer_generic_path_padding_and_group_sizes(tdq, bf16, C, g):
         assert rep["scale_max_rel"] <= 1e-6
 
 
-def test_quantizer_percentile_and_odd_rank_take_generic_kernel(tdq):
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("rank", [1, 2, 3, 5, 6, 8, 9, 11, 12, 14, 15, 17, 18, 21, 24, 27, 28, 30, 31])
+def test_quantizer_every_zero_bin_rank_on_the_fast_path(tdq, bf16, rank):
+    # zr chosen so that ceil(zr * 32) is the rank; the ranks of the other fast-path tests are left out
+    zr = (rank - 0.5) / 32.0
+    xs = [si.dc_offset_tokens(M=300, C=96), si.config1().x.reshape(-1, 64), si.edge_rows(C=64)]
+    for x in xs:
+        if bf16:
+            x = si.f32_to_bf16_bits(x)
+        ref, codes, scale = _quant_both(tdq, x, bf16, zr=zr)
+        rep = compare_quantizer(_f32(x, bf16), 32, ref, codes, scale)
+        assert rep["scale_exact_frac"] == 1.0, rep
+
+
+def test_quantizer_percentile_and_odd_rank_settings(tdq):
     x = si.config1().x.reshape(-1, 64)
     for kw in (dict(p=0.9), dict(zr=0.27), dict(zr=0.95, p=0.5)):
         ref, codes, scale = _quant_both(tdq, x, False, **kw)
