@@ -127,6 +127,7 @@ struct LinArgs {
     const float* xscale;
     int32_t row_bytes;         // I_pad / 2
     int32_t unpack_a;
+    int32_t pair_groups;       // groups of a multiple of four steps, two or more per tile: the two MMA warps take them in turn
     // fused producer only: the activations themselves and the quantizer's parameters
     const void* x;
     int64_t x_stride;          // elements between rows of x
@@ -559,8 +560,11 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
     const bool resident = a.a_resident != 0;
 
     if (t == 0) {
-        const uint32_t n_issuers = a.steps_per_grp <= 2 ? 2u : 1u;   // MMA-issuing warps
-        for (int i = 0; i < kMaxStages; ++i) { mbar_init(&c->full[i], 1); mbar_init(&c->empty[i], n_issuers); }
+        // MMA-issuing warps: two that share every ring stage (groups of one or two steps), two that take whole
+        // groups in turn (a.pair_groups), else one
+        const uint32_t n_issuers = (a.steps_per_grp <= 2 || a.pair_groups) ? 2u : 1u;
+        const uint32_t per_stage = a.steps_per_grp <= 2 ? 2u : 1u;   // of them, how many read one stage
+        for (int i = 0; i < kMaxStages; ++i) { mbar_init(&c->full[i], 1); mbar_init(&c->empty[i], per_stage); }
         for (int i = 0; i < kSlots; ++i) { mbar_init(&c->tfull[i], 1); mbar_init(&c->tempty[i], kPromoWarps); }
         for (int i = 0; i < kMaxItemBufs; ++i) {
             mbar_init(&c->a_full[i], (FUSED || a.unpack_a) ? kPromoWarps : 1);
@@ -592,6 +596,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
         if (warp < kProdWarps) {
             // ------------------------------------------------------------ producers (lane 0 issues)
             uint32_t sc = 0, s = 0, ph = 0;   // stage counter, its ring slot and phase
+            uint32_t ps = 0, pph = 0;         // paired groups: position and phase in this warp's half of the ring
+            const uint32_t n_mine = ((uint32_t)a.n_stages + 1 - (uint32_t)warp) / 2;
             uint32_t ib = 0, iu = 0;          // item buffer and its phase
             bool ok = true;
             for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
@@ -619,6 +625,28 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                 if (++ib == (uint32_t)a.n_ibuf) { ib = 0; iu ^= 1; }
                 for (int nt = part_begin(part); nt < part_begin(part + 1) && ok; ++nt) {
                     const uint8_t* b_src = a.b_blocks + (int64_t)nt * a.n_steps * kBlock;
+                    if (a.pair_groups) {
+                        // two rings: this warp feeds the MMA warp of its parity through the stages of its parity, with
+                        // the chunks of that warp's groups (group = steps_per_grp / 4 consecutive chunks of a tile)
+                        const int cpg = a.steps_per_grp / kChunk;
+                        for (int kc = 0; kc < n_chunks && ok; ++kc) {
+                            if (((kc / cpg) & 1) != warp) continue;
+                            const uint32_t st = 2 * ps + (uint32_t)warp;
+                            ok = mbar_wait_warp(&c->empty[st], pph ^ 1, c, a.status, 5u);
+                            if (!ok) break;
+                            if (lane == 0) {
+                                const uint32_t stage = ring_s + st * a.stage_bytes;
+                                mbar_expect_tx(&c->full[st], (uint32_t)kChunk * kBlock * (resident ? 1u : 2u));
+                                bulk_load(stage, b_src + (int64_t)kc * kChunk * kBlock, (uint32_t)kChunk * kBlock, &c->full[st]);
+                                if (!resident)
+                                    bulk_load(stage + kChunk * kBlock, a_src + (int64_t)kc * kChunk * kBlock,
+                                              (uint32_t)kChunk * kBlock, &c->full[st]);
+                            }
+                            __syncwarp();
+                            if (++ps == n_mine) { ps = 0; pph ^= 1; }
+                        }
+                        continue;
+                    }
                     for (int kc = 0; kc < n_chunks; ++kc, ++sc) {
                         if ((int)(sc & 1u) == warp) {
                             ok = mbar_wait_warp(&c->empty[s], ph ^ 1, c, a.status, 5u);
@@ -638,7 +666,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                     }
                 }
             }
-        } else if (warp == kMmaWarp || spg <= 2) {
+        } else if (warp == kMmaWarp || spg <= 2 || a.pair_groups) {
             // ------------------------------------------------------------ MMA issue (lane 0 issues)
             // A warp runs dependent scalar code at one instruction every few clocks, so this loop is
             // what paces the tensor pipe: everything that can be is hoisted, and the two cases are
@@ -657,10 +685,12 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
             // mode 0: one instruction per group, two warps that take the even and the odd slots (DUAL); 3: two
             // instructions per group, two warps that take the first and the second group of a chunk (DUAL2);
             // 1: groups of a multiple of four steps, so that a chunk belongs to one group and is issued as
-            // straight-line code (QUAD); 2: any other group width, one step at a time
+            // straight-line code (QUAD), by one warp when a tile has a single group; 4: the same with two or more
+            // groups per tile, which two warps take in turn, each on its own half of the ring (PAIRQ); 2: any
+            // other group width, one step at a time
             auto role = [&](auto mode_tag) {
                 constexpr int MODE = decltype(mode_tag)::value;
-                constexpr bool DUAL = MODE == 0, QUAD = MODE == 1, DUAL2 = MODE == 3;
+                constexpr bool DUAL = MODE == 0, QUAD = MODE == 1, DUAL2 = MODE == 3, PAIRQ = MODE == 4;
                 uint32_t s = 0, ph = 0, ib = 0, iu = 0;
                 bool ok = true;
                 // DUAL: this warp's two slots (me and me + 2), everything about them precomputed
@@ -671,6 +701,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                 uint32_t q_a = 1, q_b = 1;     // parity to wait for on tempty of each slot; a fresh barrier passes parity 1
                 // otherwise: one slot at a time
                 uint32_t qm = 0xFu;            // the same parities as a mask, bit = slot
+                uint32_t ps = 0, pph = 0;      // PAIRQ: position and phase in this warp's half of the ring (stages me, me + 2, ...)
+                const uint32_t n_mine = (n_stages + 1 - me) / 2;
                 for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
                     const int part = item % a.n_parts;
                     const int n_tiles = part_begin(part + 1) - part_begin(part);
@@ -681,7 +713,36 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                         uint32_t slot = 0;
                         bool slot_ready = false;   // the early answer about the next slot, if it was yes
                         uint32_t a_lo = ares_lo;   // resident: walks through the item's A blocks
+                        uint32_t grp = 0;          // PAIRQ: group of the tile this chunk belongs to
                         for (int k0 = 0; k0 < n_steps && ok; k0 += kChunk) {
+                            if (PAIRQ) {
+                                // A group is spg / 4 consecutive chunks and belongs to the warp of its parity, which has
+                                // every second ring stage to itself (fed by the producer warp of the same parity): two
+                                // independent rings, so neither warp ever looks at a barrier of the other's.
+                                if ((grp & 1u) == me) {
+                                    const uint32_t st = 2 * ps + me, gslot = grp & (kSlots - 1);
+                                    ok = mbar_wait_warp(&c->full[st], pph, c, a.status, 4u);
+                                    if (!ok) break;
+                                    if (sub == 0 && !__all_sync(0xffffffffu, mbar_test_s(tempty_s + gslot * 8, (qm >> gslot) & 1u))) {
+                                        ok = mbar_wait_warp(&c->tempty[gslot], (qm >> gslot) & 1u, c, a.status, 3u);
+                                        if (!ok) break;
+                                    }
+                                    tc_fence_after();
+                                    const uint32_t b_st = ring_lo + st * stage_step;
+                                    mma_issue4_if<I8>(lane0, tmem_base + gslot * kBN, resident ? a_lo : b_st + a_in_stage, b_st,
+                                                      sub == 0 ? 0u : 1u);
+                                    if (sub + kChunk == spg) {
+                                        mma_commit_if(lane0, tfull_s + gslot * 8);
+                                        qm ^= 1u << gslot;
+                                    }
+                                    mma_commit_if(lane0, empty_s + st * 8);
+                                    if (++ps == n_mine) { ps = 0; pph ^= 1; }
+                                }
+                                sub += kChunk;
+                                if (sub == spg) { sub = 0; ++grp; }
+                                if (resident) a_lo += kChunk * (kBlock >> 4);
+                                continue;
+                            }
                             ok = mbar_wait_warp(&c->full[s], ph, c, a.status, 4u);
                             if (!ok) break;
                             const uint32_t b_lo = ring_lo + s * stage_step;
@@ -773,6 +834,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
             };
             if (spg == 1) role(std::integral_constant<int, 0>{});
             else if (spg == 2) role(std::integral_constant<int, 3>{});
+            else if (a.pair_groups) role(std::integral_constant<int, 4>{});
             else if (spg % kChunk == 0) role(std::integral_constant<int, 1>{});
             else role(std::integral_constant<int, 2>{});
         }
@@ -1335,6 +1397,7 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
     a.half_strips = half_strips ? 1 : 0;
     a.out_scale = i8 ? 0.00390625f : 262144.0f;
     a.xcodes = xcodes; a.xscale = xscale; a.row_bytes = e.row_bytes; a.unpack_a = unpack_a ? 1 : 0;
+    a.pair_groups = (a.steps_per_grp % kChunk == 0 && a.Kg >= 2) ? 1 : 0;
     a.x = fx ? fx->x : nullptr;
     a.x_stride = fx ? fx->row_stride : 0;
     a.seven_tau = fx ? fx->seven_tau : 0.0f;
