@@ -625,7 +625,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                 if (++ib == (uint32_t)a.n_ibuf) { ib = 0; iu ^= 1; }
                 for (int nt = part_begin(part); nt < part_begin(part + 1) && ok; ++nt) {
                     const uint8_t* b_src = a.b_blocks + (int64_t)nt * a.n_steps * kBlock;
-                    if (a.pair_groups) {
+                    if (I8 && a.pair_groups) {   // (wide groups always take the integer instruction)
                         // two rings: this warp feeds the MMA warp of its parity through the stages of its parity, with
                         // the chunks of that warp's groups (group = steps_per_grp / 4 consecutive chunks of a tile)
                         const int cpg = a.steps_per_grp / kChunk;
@@ -666,7 +666,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                     }
                 }
             }
-        } else if (warp == kMmaWarp || spg <= 2 || a.pair_groups) {
+        } else if (warp == kMmaWarp || spg <= 2 || (I8 && a.pair_groups)) {
             // ------------------------------------------------------------ MMA issue (lane 0 issues)
             // A warp runs dependent scalar code at one instruction every few clocks, so this loop is
             // what paces the tensor pipe: everything that can be is hoisted, and the two cases are
@@ -834,7 +834,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
             };
             if (spg == 1) role(std::integral_constant<int, 0>{});
             else if (spg == 2) role(std::integral_constant<int, 3>{});
-            else if (a.pair_groups) role(std::integral_constant<int, 4>{});
+            else if (I8 && a.pair_groups) role(std::integral_constant<int, 4>{});
             else if (spg % kChunk == 0) role(std::integral_constant<int, 1>{});
             else role(std::integral_constant<int, 2>{});
         }
@@ -1397,7 +1397,7 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
     a.half_strips = half_strips ? 1 : 0;
     a.out_scale = i8 ? 0.00390625f : 262144.0f;
     a.xcodes = xcodes; a.xscale = xscale; a.row_bytes = e.row_bytes; a.unpack_a = unpack_a ? 1 : 0;
-    a.pair_groups = (a.steps_per_grp % kChunk == 0 && a.Kg >= 2) ? 1 : 0;
+    a.pair_groups = (i8 && a.steps_per_grp % kChunk == 0 && a.Kg >= 2) ? 1 : 0;
     a.x = fx ? fx->x : nullptr;
     a.x_stride = fx ? fx->row_stride : 0;
     a.seven_tau = fx ? fx->seven_tau : 0.0f;
