@@ -43,7 +43,7 @@ L2_BYTES = 126 * 2 ** 20
 
 # DRAM bytes (read + write) of one w4a4_gemm_kernel launch on cfg4 from the ncu capture summarised in
 # profiles/w4a4_gemm_kernel_cfg4.md; reported only for that workload and output type.
-GEMM_DRAM_TRAFFIC_CFG4 = 179.2e6
+GEMM_DRAM_TRAFFIC_CFG4 = 179.0e6
 
 
 def load_peaks():
