@@ -1,0 +1,216 @@
+"""GPU parity at the configured sizes: every row of the large single-layer workloads, every layer of the
+32-layer sweep at its batch size, a constructed set of rounding-boundary inputs, channel-major input through
+the linear layer, and row shards against the unsharded call.  Everything goes through the C ABI (ctypes
+binding of libtdq.so) and is compared with the CPU oracle under the rules of parity_utils."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth_inputs as si
+from parity_utils import compare_quantizer, compare_y, to_cuda, unpack_codes
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def tdq():
+    from paper_2604_16855_b200 import tdq
+    return tdq
+
+
+def _f32(x_np, bf16):
+    return si.bf16_bits_to_f32(x_np) if bf16 else x_np
+
+
+# ---------------------------------------------------------------------------------------
+# the two large single-layer workloads: quantizer -> linear layer, every row against the oracle
+
+@pytest.mark.parametrize("idx", [3, 4])
+def test_large_workloads_every_row(tdq, idx):
+    case = si.config(idx)
+    x = case.x.reshape(-1, case.C)
+    K = case.C // 32
+    xt = to_cuda(x, bf16=case.x_is_bf16)
+    wc, ws = tdq.quantize_weight(to_cuda(case.w))
+    codes, scale = tdq.quantize_act(xt)
+    wsp = tdq.linear_workspace(x.shape[0], case.C, case.O, 32, "cuda")
+    y = tdq.w4a4_linear(codes, scale, wc, ws, workspace=wsp)
+    st, detail = tdq.workspace_status(wsp)
+    assert st == tdq.OK, "device wait ran out: 0x%x" % detail
+    xa = oracle.quantize_act(x)
+    wq = oracle.quantize_weight(case.w)
+    np.testing.assert_array_equal(codes.cpu().numpy(), xa["codes"])
+    np.testing.assert_array_equal(scale.cpu().numpy(), xa["scale"])
+    np.testing.assert_array_equal(wc.cpu().numpy(), wq["codes"])
+    ref = oracle.w4a4_linear(xa["codes"], xa["scale"], wq["codes"], wq["scale"])
+    worst, strict = compare_y(y.cpu().numpy(), ref, K)
+    print("cfg%d, all %d rows: worst err/tol %.3f, %.6f of outputs within 1e-5 relative" % (idx, x.shape[0], worst, strict))
+    assert strict > 0.99
+
+
+# ---------------------------------------------------------------------------------------
+# the 32-layer sweep at batch 8: every layer, quantizer and linear layer, and the fused call where it applies
+
+@pytest.mark.parametrize("layer", list(range(32)))
+def test_sweep_every_layer_at_batch_8(tdq, layer):
+    case = si.config5_layer(layer, batch=8)
+    x = case.x.reshape(-1, case.C)
+    M, K = x.shape[0], case.C // 32
+    xt = to_cuda(x, bf16=True)
+    wc, ws = tdq.quantize_weight(to_cuda(case.w))
+    codes, scale = tdq.quantize_act(xt)
+    wsp = tdq.linear_workspace(M, case.C, case.O, 32, "cuda")
+    y = tdq.w4a4_linear(codes, scale, wc, ws, workspace=wsp)
+    st, detail = tdq.workspace_status(wsp)
+    assert st == tdq.OK, "device wait ran out: 0x%x" % detail
+    xa = oracle.quantize_act(x)
+    wq = oracle.quantize_weight(case.w)
+    rep = compare_quantizer(_f32(x, True), 32, xa, codes.cpu().numpy(), scale.cpu().numpy())
+    assert rep["code_mismatch"] == 0 and rep["scale_exact_frac"] == 1.0, rep
+    ref = oracle.w4a4_linear(xa["codes"], xa["scale"], wq["codes"], wq["scale"])
+    worst, strict = compare_y(y.cpu().numpy(), ref, K)
+    assert strict > 0.99
+    if case.C <= 768:                            # the fused call keeps a row block's operand in shared memory
+        yf = tdq.quant_linear_fused(xt, wc, ws)
+        compare_y(yf.cpu().numpy(), ref, K)
+    else:
+        with pytest.raises(tdq.TdqError) as e:
+            tdq.quant_linear_fused(xt, wc, ws)
+        assert e.value.code == tdq.ERR_UNSUPPORTED
+    print("layer %d (%d x %d -> %d): worst err/tol %.3f" % (layer, M, case.C, case.O, worst))
+
+
+# ---------------------------------------------------------------------------------------
+# rounding boundaries: inputs placed on and next to the half-integers of x / Delta
+
+def _boundary_rows_fp32(n_rows, seed):
+    """Rows of three groups whose step is set by the group's largest element c (a random binary32 mantissa and
+    exponent): the other elements sit at (k + 1/2) * fl(c / 7), k = -7 .. 6, moved by 0, +-1 and +-2 ulp."""
+    rng = np.random.default_rng(seed)
+    c = (rng.uniform(1.0, 2.0, n_rows) * 2.0 ** rng.integers(-20, 20, n_rows)).astype(np.float32)
+    delta = (c / np.float32(7.0)).astype(np.float32)
+    vals = []
+    for k in range(-7, 7):
+        base = (np.float32(k + 0.5) * delta).astype(np.float32)
+        for n in (-2, -1, 0, 1, 2):
+            v = base.copy()
+            for _ in range(abs(n)):
+                v = np.nextafter(v, np.float32(np.inf if n > 0 else -np.inf), dtype=np.float32)
+            vals.append(v)
+    vals = np.stack(vals, 1)                       # [n_rows, 70]
+    x = np.zeros((n_rows, 96), np.float32)
+    for g in range(3):
+        x[:, 32 * g] = c * (1 if g != 1 else -1)   # the group's largest magnitude
+        take = vals[:, 24 * g: 24 * g + 24] if g < 2 else vals[:, 46:70]
+        x[:, 32 * g + 1: 32 * g + 1 + take.shape[1]] = take
+        x[:, 32 * g + 25: 32 * g + 32] = (rng.uniform(-1, 1, (n_rows, 7)).astype(np.float32) * c[:, None])
+    return x
+
+
+def _boundary_rows_zero_bin(n_rows, seed, bf16):
+    """Groups in which the zero-bin bound is the active one: six small elements, the threshold element thr, odd
+    multiples of thr (the half-integers of x / Delta, since Delta = 2 thr when 14 thr is exact) and their
+    neighbours, and a few large elements that keep the other two bounds away."""
+    rng = np.random.default_rng(seed)
+    mant = rng.integers(8, 16, n_rows).astype(np.float32) if bf16 else rng.uniform(1.0, 2.0, n_rows).astype(np.float32)
+    thr = (mant * np.float32(2.0) ** rng.integers(-12, 8, n_rows).astype(np.float32)).astype(np.float32)
+    x = np.zeros((n_rows, 32), np.float32)
+    x[:, :6] = thr[:, None] * rng.uniform(0.05, 0.9, (n_rows, 6)).astype(np.float32)
+    x[:, 6] = thr
+    odd = np.array([3, -3, 5, -5, 7, -7, 9, -9, 11, -11, 13, -13], np.float32)
+    x[:, 7:19] = thr[:, None] * odd[None, :]
+    nb = x[:, 7:13].copy()
+    step = np.float32(2.0 ** -7) if bf16 else np.float32(2.0 ** -23)
+    x[:, 19:25] = nb * (np.float32(1.0) + step)    # one unit in the last place above (bf16) or one ulp (fp32)
+    x[:, 25:29] = x[:, 7:11] * (np.float32(1.0) - step)
+    x[:, 29:32] = thr[:, None] * np.array([40.0, -60.0, 50.0], np.float32)[None, :]
+    perm = rng.permuted(np.tile(np.arange(32), (n_rows, 1)), axis=1)
+    return np.take_along_axis(x, perm, axis=1)
+
+
+@pytest.mark.parametrize("kind", ["fp32_base", "fp32_zero_bin", "bf16_zero_bin"])
+def test_quotients_on_rounding_boundaries(tdq, kind):
+    bf16 = kind.startswith("bf16")
+    if kind == "fp32_base":
+        x = _boundary_rows_fp32(6000, 5)
+        settings = [dict(flags=0), dict(flags=3)]
+    else:
+        x = _boundary_rows_zero_bin(20000, 9 if bf16 else 8, bf16)
+        settings = [dict(flags=3), dict(flags=2)]
+    xin = si.f32_to_bf16_bits(x) if bf16 else x
+    xf = _f32(xin, bf16)
+    for kw in settings:
+        ref = oracle.quantize_act(xin, **kw)
+        codes, scale = tdq.quantize_act(to_cuda(xin, bf16=bf16), tdq.act_params(**kw))
+        torch.cuda.synchronize()
+        rep = compare_quantizer(xf, 32, ref, codes.cpu().numpy(), scale.cpu().numpy())
+        # how adversarial the set is: elements whose quotient lies within 4 ulp of a half-integer
+        d = np.repeat(ref["scale"].astype(np.float64), 32, axis=1)
+        cl = np.repeat(ref["clip"].astype(np.float64), 32, axis=1)
+        r = np.clip(xf.astype(np.float64), -cl, cl) / d
+        near = np.abs(np.abs(r - np.floor(r)) - 0.5) <= 4 * 2.0 ** -23 * np.maximum(np.abs(r), 1.0)
+        print("%s %s: %d elements, %.1f %% within 4 ulp of a rounding boundary, %d code mismatches, scales exact %.6f"
+              % (kind, kw, near.size, 100.0 * near.mean(), rep["code_mismatch"], rep["scale_exact_frac"]))
+        assert near.mean() > 0.05
+        assert rep["code_mismatch"] == 0 and rep["scale_exact_frac"] == 1.0
+
+
+# ---------------------------------------------------------------------------------------
+# channel-major input through the linear layer (a 1 x 1 convolution), against the oracle
+
+@pytest.mark.parametrize("B,C,H,W,O,bf16", [(2, 64, 9, 16, 96, True), (1, 320, 24, 24, 320, True), (2, 128, 8, 8, 40, False)])
+def test_channel_major_quantizer_feeds_the_linear_layer(tdq, B, C, H, W, O, bf16):
+    rng = np.random.default_rng(B * 100 + C + O)
+    sig = np.exp(rng.normal(0.0, 0.7, size=(B, 1, H, W)))
+    x = (rng.normal(size=(B, C, H, W)) * sig).astype(np.float32)
+    x[rng.random((B, C, H, W)) < 0.02] *= 30.0
+    xin = si.f32_to_bf16_bits(x) if bf16 else x
+    w = si.weights(rng, O, C)
+    bias = rng.standard_normal(O).astype(np.float32) * 0.1
+    codes, scale = tdq.quantize_act_nchw(to_cuda(xin, bf16=bf16))
+    wc, ws = tdq.quantize_weight(to_cuda(w))
+    y = tdq.w4a4_linear(codes, scale, wc, ws, to_cuda(bias))          # [B*H*W, O], token (b, h, w) in row (b*H + h)*W + w
+    xa = oracle.quantize_act_nchw(xin)
+    wq = oracle.quantize_weight(w)
+    np.testing.assert_array_equal(codes.cpu().numpy(), xa["codes"])
+    np.testing.assert_array_equal(scale.cpu().numpy(), xa["scale"])
+    ref = oracle.w4a4_linear(xa["codes"], xa["scale"], wq["codes"], wq["scale"], bias=bias)
+    compare_y(y.cpu().numpy(), ref, C // 32 + 1)
+    # the rows are in token order: one position checked by plain indexing against the dequantized operands
+    b, h, wq_pos = B - 1, H // 2, W - 1
+    t = (b * H + h) * W + wq_pos
+    xq = unpack_codes(xa["codes"])[t].astype(np.float64) * np.repeat(xa["scale"][t].astype(np.float64), 32)
+    wd = unpack_codes(wq["codes"]).astype(np.float64) * wq["scale"].astype(np.float64)[:, None]
+    np.testing.assert_allclose(y.cpu().numpy()[t], wd @ xq + bias, rtol=1e-4, atol=1e-5 * np.abs(wd @ xq).max())
+    # and the dequantized token is the token at (b, :, h, w) of the map, within half a step per channel
+    xf = _f32(xin, bf16)
+    assert (np.abs(xq[:C] - np.clip(xf[b, :, h, wq_pos], -np.repeat(xa["clip"][t], 32)[:C], np.repeat(xa["clip"][t], 32)[:C]))
+            <= 0.5000001 * np.repeat(xa["scale"][t], 32)[:C]).all()
+
+
+# ---------------------------------------------------------------------------------------
+# row shards: two ranges of rows through the path separately equal the unsharded call bit for bit
+
+@pytest.mark.parametrize("idx,rows,split", [(2, 5000, 2176), (3, 3000, 1409), (1, 256, 100)])
+def test_row_shards_equal_the_unsharded_call(tdq, idx, rows, split):
+    case = si.config(idx)
+    x = case.x.reshape(-1, case.C)[:rows]
+    xt = to_cuda(x, bf16=case.x_is_bf16)
+    wc, ws = tdq.quantize_weight(to_cuda(case.w))
+    bias = torch.linspace(-0.5, 0.5, case.O, device="cuda")
+
+    def path(xpart):
+        codes, scale = tdq.quantize_act(xpart)
+        return codes, scale, tdq.w4a4_linear(codes, scale, wc, ws, bias)
+
+    c_all, s_all, y_all = path(xt)
+    c0, s0, y0 = path(xt[:split])
+    c1, s1, y1 = path(xt[split:].contiguous())
+    assert torch.equal(torch.cat([c0, c1]), c_all)
+    assert torch.equal(torch.cat([s0, s1]).view(torch.int32), s_all.view(torch.int32))
+    assert torch.equal(torch.cat([y0, y1]).view(torch.int32), y_all.view(torch.int32))
+    if case.C <= 768:
+        yf0 = tdq.quant_linear_fused(xt[:split], wc, ws, bias)
+        yf1 = tdq.quant_linear_fused(xt[split:].contiguous(), wc, ws, bias)
+        assert torch.equal(torch.cat([yf0, yf1]).view(torch.int32), y_all.view(torch.int32))

@@ -34,10 +34,10 @@ def test_static_scratch_entry_matches_workspace_entry_twice_in_a_row():
         y = torch.full((rows, case.O), float("nan"), device="cuda")
         tdq.w4a4_linear_static(xc, xs, wc, ws, bias, y=y, wait=True)
         torch.cuda.synchronize()
-        a, b = y.cpu().numpy().astype(np.float64), y_ref.cpu().numpy().astype(np.float64)
-        assert np.isfinite(a).all()
-        # the tolerance the other output tests use against the oracle; here both sides run the same kernels
-        assert (np.abs(a - b) <= 1e-5 * np.abs(b) + 1e-30).all()
+        assert torch.isfinite(y).all()
+        # both entries run the same kernels on the same operand blocks, so the outputs agree bit for bit (which is
+        # inside any tolerance the other output tests use)
+        assert torch.equal(y.view(torch.int32), y_ref.view(torch.int32))
 
 
 def test_static_scratch_entry_refuses_what_does_not_fit():
