@@ -12,9 +12,14 @@
  *     default stream) and the call returns without waiting for it.
  *   - Arguments are checked on the host before anything is launched.  A bad argument
  *     returns an error code and launches nothing.  Nothing throws, aborts or traps.
- *   - Kernels whose threads wait on each other give every wait an iteration limit.  A
- *     wait that runs out writes a code into the call's workspace and the kernel returns;
- *     tdq_workspace_status() reads that word back.
+ *   - Kernels whose threads wait on each other give every wait a limit of about a second.  A
+ *     wait that runs out records a code and the kernel returns with part of its output
+ *     unwritten.  The linear-layer calls record it in the call's workspace, read back by
+ *     tdq_workspace_status(); the quantizer calls, which have no workspace, in one word per
+ *     device, read back (and cleared) by tdq_quantize_status().
+ *   - The library allocates no device memory.  tdq_quant_linear_host creates two streams and
+ *     a few events per device on first use and keeps them for the life of the process; no
+ *     other call creates CUDA objects.
  *   - Non-finite inputs (NaN, Inf) give unspecified codes; they never fault.
  *
  * Notation (the paper's): M = B*N tokens, C = I input channels, O output channels,
@@ -254,6 +259,30 @@ size_t tdq_linear_workspace_bytes(int64_t M, int64_t I_pad, int64_t O, int32_t g
  * bits 0-7 name the wait that gave up, bits 8-31 the tile index.
  */
 tdq_status tdq_workspace_status(const void* workspace, void* cuda_stream, uint32_t* detail /* HOST */);
+
+/*
+ * Waits for cuda_stream, then reads the word in which the quantizer kernels of the current device
+ * (tdq_quantize_act and its variants, which have no workspace) record a bounded wait that ran out:
+ * TDQ_OK, or TDQ_ERR_DEVICE_TIMEOUT when one did since the last query (codes and scales of that
+ * call are then incomplete).  detail (HOST, nullable) receives the raw word: bits 0-7 name the wait
+ * (12 the tile producer, 13 a consumer warp, 14 the self-test), bits 8-31 the thread block.  A
+ * non-zero word is cleared by the query.  The word is shared by all streams of the device.
+ */
+tdq_status tdq_quantize_status(void* cuda_stream, uint32_t* detail /* HOST */);
+
+/*
+ * Self-test of the bounded waits (no counterpart in the paper): one warp waits, with the kernels' own
+ * wait routine and a limit of limit_cycles SM clocks (1000 .. 2e9), on a barrier that nobody arrives
+ * on, gives up, records its code and returns; no copy or tensor-core operation is in flight when it
+ * leaves, so the device stays usable.
+ *   which == 0: the linear layer's routine; the code (15) goes to the status word of `workspace`
+ *               (16-byte aligned, at least 256 bytes), which the call clears first; read it with
+ *               tdq_workspace_status().
+ *   which == 1: the quantizer's routine; the code (14) goes to the per-device word that
+ *               tdq_quantize_status() reads; workspace is ignored.
+ * The call is asynchronous on cuda_stream like every other one.
+ */
+tdq_status tdq_selftest_wait_timeout(int32_t which, int64_t limit_cycles, void* workspace, void* cuda_stream);
 
 /* Static description of a status code. */
 const char* tdq_status_string(tdq_status s);

@@ -23,7 +23,8 @@ ENABLE_C1, ENABLE_C2, POW2_STEP = 1, 2, 4
 # every symbol include/tdq.h declares
 EXPORTS = ["tdq_default_act_params", "tdq_quantize_act", "tdq_quantize_weight", "tdq_w4a4_linear",
            "tdq_quant_linear_fused", "tdq_quant_linear_host", "tdq_quantize_act_nchw", "tdq_quantize_act_fixed", "tdq_w4a4_linear_pow2", "tdq_linear_workspace_bytes",
-           "tdq_workspace_status", "tdq_status_string", "tdq_kernel_launch_count", "tdq_w4a4_linear_static"]
+           "tdq_workspace_status", "tdq_status_string", "tdq_kernel_launch_count", "tdq_w4a4_linear_static",
+           "tdq_quantize_status", "tdq_selftest_wait_timeout"]
 
 
 class ActParams(ctypes.Structure):
@@ -61,6 +62,10 @@ _lib.tdq_linear_workspace_bytes.argtypes = [_i64, _i64, _i64, _i32]
 _lib.tdq_linear_workspace_bytes.restype = _sz
 _lib.tdq_workspace_status.argtypes = [_vp, _vp, ctypes.POINTER(ctypes.c_uint32)]
 _lib.tdq_workspace_status.restype = ctypes.c_int
+_lib.tdq_quantize_status.argtypes = [_vp, ctypes.POINTER(ctypes.c_uint32)]
+_lib.tdq_quantize_status.restype = ctypes.c_int
+_lib.tdq_selftest_wait_timeout.argtypes = [_i32, _i64, _vp, _vp]
+_lib.tdq_selftest_wait_timeout.restype = ctypes.c_int
 _lib.tdq_status_string.argtypes = [ctypes.c_int]
 _lib.tdq_status_string.restype = ctypes.c_char_p
 _lib.tdq_kernel_launch_count.argtypes = []
@@ -196,6 +201,35 @@ def quantize_weight(w: torch.Tensor, pad_to: int = 32, *, wcodes=None, wscale=No
     return wcodes, wscale
 
 
+def _check_operands(named, y=None):
+    """The layout the C ABI assumes but cannot see: dtype, contiguity, one common device; y may have a row pitch
+    but its columns must be adjacent.  `named` is a list of (name, tensor or None, dtype).  Returns the device."""
+    dev = None
+    for name, t, dt in named:
+        if t is None:
+            continue
+        if t.dtype != dt:
+            raise TypeError("%s must be %s, got %s" % (name, dt, t.dtype))
+        if not t.is_contiguous():
+            raise ValueError("%s must be contiguous" % name)
+        if dev is None:
+            dev = t.device
+        elif t.device != dev:
+            raise ValueError("%s is on %s, the other operands on %s" % (name, t.device, dev))
+    if y is not None:
+        if y.dim() != 2 or (y.shape[1] > 1 and y.stride(1) != 1):
+            raise ValueError("y must be a matrix whose columns are adjacent in memory")
+        if dev is not None and y.device != dev:
+            raise ValueError("y is on %s, the operands on %s" % (y.device, dev))
+    return dev
+
+
+def _linear_operands(xcodes, xscale, wcodes, wscale, bias, y, workspace=None, acc_debug=None):
+    return _check_operands([("xcodes", xcodes, torch.uint8), ("xscale", xscale, torch.float32), ("wcodes", wcodes, torch.uint8),
+                            ("wscale", wscale, torch.float32), ("bias", bias, torch.float32),
+                            ("workspace", workspace, torch.uint8), ("acc_debug", acc_debug, torch.int32)], y)
+
+
 def linear_workspace(M, I_pad, O, g, device) -> torch.Tensor:
     n = int(_lib.tdq_linear_workspace_bytes(M, I_pad, O, g))
     return torch.zeros((n,), dtype=torch.uint8, device=device)
@@ -212,9 +246,11 @@ def w4a4_linear(xcodes, xscale, wcodes, wscale, bias=None, *, g=32, out_dtype=to
         y = torch.empty((M, O), dtype=out_dtype, device=xcodes.device)
     if workspace is None:
         workspace = linear_workspace(M, I_pad, O, g, xcodes.device)
-    _check(_lib.tdq_w4a4_linear(_ptr(xcodes), _ptr(xscale), _ptr(wcodes), _ptr(wscale), _ptr(bias), M, I_pad, O, g,
-                                _ptr(y), _dtype_id(y), y.stride(0) if M > 0 else O, _ptr(acc_debug),
-                                _ptr(workspace), workspace.numel(), _stream(xcodes)), "tdq_w4a4_linear")
+    dev = _linear_operands(xcodes, xscale, wcodes, wscale, bias, y, workspace, acc_debug)
+    with torch.cuda.device(dev):        # the library works on the current device
+        _check(_lib.tdq_w4a4_linear(_ptr(xcodes), _ptr(xscale), _ptr(wcodes), _ptr(wscale), _ptr(bias), M, I_pad, O, g,
+                                    _ptr(y), _dtype_id(y), y.stride(0) if M > 0 else O, _ptr(acc_debug),
+                                    _ptr(workspace), workspace.numel(), _stream(xcodes)), "tdq_w4a4_linear")
     return y
 
 
@@ -228,9 +264,11 @@ def w4a4_linear_pow2(xcodes, xscale, wcodes, wscale, bias=None, *, g=32, out_dty
         y = torch.empty((M, O), dtype=out_dtype, device=xcodes.device)
     if workspace is None:
         workspace = linear_workspace(M, I_pad, O, g, xcodes.device)
-    _check(_lib.tdq_w4a4_linear_pow2(_ptr(xcodes), _ptr(xscale), _ptr(wcodes), _ptr(wscale), _ptr(bias), M, I_pad, O, g,
-                                     _ptr(y), _dtype_id(y), y.stride(0) if M > 0 else O, _ptr(workspace),
-                                     workspace.numel(), _stream(xcodes)), "tdq_w4a4_linear_pow2")
+    dev = _linear_operands(xcodes, xscale, wcodes, wscale, bias, y, workspace)
+    with torch.cuda.device(dev):
+        _check(_lib.tdq_w4a4_linear_pow2(_ptr(xcodes), _ptr(xscale), _ptr(wcodes), _ptr(wscale), _ptr(bias), M, I_pad, O, g,
+                                         _ptr(y), _dtype_id(y), y.stride(0) if M > 0 else O, _ptr(workspace),
+                                         workspace.numel(), _stream(xcodes)), "tdq_w4a4_linear_pow2")
     return y
 
 
@@ -245,9 +283,11 @@ def w4a4_linear_static(xcodes, xscale, wcodes, wscale, bias=None, *, g=32, y, wa
     _need_cuda(xcodes, xscale, wcodes, wscale, bias, y)
     M, half = xcodes.shape
     O = wcodes.shape[0]
-    _check(_lib.tdq_w4a4_linear_static(_ptr(xcodes), _ptr(xscale), _ptr(wcodes), _ptr(wscale), _ptr(bias), M, half * 2,
-                                       O, g, _ptr(y), _dtype_id(y), y.stride(0) if M > 0 else O, 1 if wait else 0,
-                                       _stream(xcodes)), "tdq_w4a4_linear_static")
+    dev = _linear_operands(xcodes, xscale, wcodes, wscale, bias, y)
+    with torch.cuda.device(dev):        # the scratch array is looked up on the current device
+        _check(_lib.tdq_w4a4_linear_static(_ptr(xcodes), _ptr(xscale), _ptr(wcodes), _ptr(wscale), _ptr(bias), M, half * 2,
+                                           O, g, _ptr(y), _dtype_id(y), y.stride(0) if M > 0 else O, 1 if wait else 0,
+                                           _stream(xcodes)), "tdq_w4a4_linear_static")
     return y
 
 
@@ -265,9 +305,16 @@ def quant_linear_fused(x, wcodes, wscale, bias=None, params: ActParams | None = 
     if workspace is None:
         workspace = linear_workspace(M, wcodes.shape[1] * 2, O, p.group_size, x.device)
     stride = x2.stride(0) if M > 1 else C
-    _check(_lib.tdq_quant_linear_fused(_ptr(x2), _dtype_id(x2), 1, M, C, stride, ctypes.byref(p), _ptr(wcodes),
-                                       _ptr(wscale), _ptr(bias), O, _ptr(y), _dtype_id(y), y.stride(0),
-                                       _ptr(workspace), workspace.numel(), _stream(x)), "tdq_quant_linear_fused")
+    if x2.dim() != 2 or (C > 1 and x2.stride(1) != 1):
+        raise ValueError("the channels of x must be adjacent in memory")
+    dev = _check_operands([("wcodes", wcodes, torch.uint8), ("wscale", wscale, torch.float32), ("bias", bias, torch.float32),
+                           ("workspace", workspace, torch.uint8)], y)
+    if x2.device != dev:
+        raise ValueError("x is on %s, the weights on %s" % (x2.device, dev))
+    with torch.cuda.device(dev):
+        _check(_lib.tdq_quant_linear_fused(_ptr(x2), _dtype_id(x2), 1, M, C, stride, ctypes.byref(p), _ptr(wcodes),
+                                           _ptr(wscale), _ptr(bias), O, _ptr(y), _dtype_id(y), y.stride(0),
+                                           _ptr(workspace), workspace.numel(), _stream(x)), "tdq_quant_linear_fused")
     return y
 
 
@@ -301,3 +348,18 @@ def workspace_status(workspace: torch.Tensor):
     detail = ctypes.c_uint32(0)
     st = _lib.tdq_workspace_status(_ptr(workspace), _stream(workspace), ctypes.byref(detail))
     return int(st), int(detail.value)
+
+
+def quantize_status(device=None):
+    """(status, detail) of the quantizer kernels' bounded waits on the current stream's device; clears the word."""
+    detail = ctypes.c_uint32(0)
+    st = _lib.tdq_quantize_status(ctypes.c_void_p(torch.cuda.current_stream(device).cuda_stream), ctypes.byref(detail))
+    return st, detail.value
+
+
+def selftest_wait_timeout(which: int, limit_cycles: int, workspace: torch.Tensor | None = None):
+    """Makes one bounded wait run out (see tdq.h); the status is read with workspace_status / quantize_status."""
+    ws = ctypes.c_void_p(workspace.data_ptr()) if workspace is not None else None
+    dev = workspace.device if workspace is not None else None
+    _check(_lib.tdq_selftest_wait_timeout(which, limit_cycles, ws, ctypes.c_void_p(torch.cuda.current_stream(dev).cuda_stream)),
+           "tdq_selftest_wait_timeout")

@@ -65,9 +65,24 @@ extern "C" tdq_status tdq_quant_linear_host(const void* x_host, tdq_dtype x_dtyp
     if (B < 0 || N < 0 || C <= 0 || O <= 0) return TDQ_ERR_INVALID_ARG;
     if (x_dtype != TDQ_F32 && x_dtype != TDQ_BF16) return TDQ_ERR_INVALID_ARG;
     if (y_dtype != TDQ_F32 && y_dtype != TDQ_BF16) return TDQ_ERR_INVALID_ARG;
-    if (p->group_size <= 0) return TDQ_ERR_INVALID_ARG;
+    // every check of the two calls that does not depend on a chunk's pointers is made here, before anything is
+    // queued: a refusal must leave the streams untouched
+    tdq_status chk = check_act_args(x_dev, x_dtype, B, N, C, C, p);
+    if (chk != TDQ_OK) return chk;
+    if (!wcodes || !wscale || !workspace) return wcodes && wscale ? TDQ_ERR_WORKSPACE : TDQ_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(wcodes) % 16 || reinterpret_cast<uintptr_t>(workspace) % 16 ||
+        reinterpret_cast<uintptr_t>(codes_dev) % 16)
+        return TDQ_ERR_ALIGNMENT;
     const int64_t M = B * N;
     if (M == 0) return TDQ_OK;
+    {
+        const int64_t g0 = p->group_size, Ip = (C + g0 - 1) / g0 * g0;
+        int64_t rp = (M + kHostChunks - 1) / kHostChunks;
+        rp = (rp + 127) / 128 * 128;
+        if (((Ip / 2) * rp) % 16) return TDQ_ERR_ALIGNMENT;        // every chunk's codes must start 16-byte aligned
+        chk = linear_check_shape(rp < M ? rp : M, Ip, O, p->group_size, workspace_bytes);
+        if (chk != TDQ_OK) return chk;
+    }
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
     HostPipe* hp = host_pipe();
     if (!hp) return TDQ_ERR_CUDA;

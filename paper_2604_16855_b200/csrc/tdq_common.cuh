@@ -37,10 +37,37 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
                        const float* wscale, const float* bias, int64_t M, int64_t I_pad, int64_t O, int32_t group_size,
                        void* y, tdq_dtype y_dtype, int64_t y_row_stride, int32_t* acc_debug, void* workspace,
                        size_t workspace_bytes, void* cuda_stream, int pow2_steps);
+// The shape, plan and workspace-size checks of tdq_w4a4_linear without its pointers: what a caller that chains
+// several calls needs to know before it enqueues the first one (tdq_linear.cu).
+tdq_status linear_check_shape(int64_t M, int64_t I_pad, int64_t O, int32_t group_size, size_t workspace_bytes);
 // Argument checks of the quantizer and its fast-path conditions (tdq_quantize_act.cu).
 tdq_status check_act_args(const void* x, tdq_dtype dt, int64_t B, int64_t N, int64_t C, int64_t stride,
                           const tdq_act_params* p);
 bool act_fast_path_ok(const void* x, tdq_dtype dt, int64_t C, int64_t stride, const tdq_act_params* p);
+
+// One warp waits, with the quantizer's ring-wait routine and the given cycle limit, on a barrier nobody arrives on
+// (tdq_selftest_wait_timeout; tdq_quantize_act.cu).
+tdq_status act_wait_selftest(long long limit_cycles, cudaStream_t stream);
+
+// Bookkeeping kept per device (a process may drive several): the SM count of the current device, looked up once
+// for each, and which devices a kernel's opt-in to large dynamic shared memory has been made on (the attribute
+// belongs to the device's context).  Lock-free: a lost race only repeats an idempotent call.
+constexpr int kMaxDevices = 64;
+inline int current_device_sm_count(int* device = nullptr) {
+    static std::atomic<int> cache[kMaxDevices];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
+    if (device) *device = dev;
+    int n = cache[dev].load(std::memory_order_relaxed);
+    if (n == 0) {
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+        cache[dev].store(n, std::memory_order_relaxed);
+    }
+    return n;
+}
+// true once `done` has the device's bit; the caller sets the attribute when this returns false and then calls mark
+inline bool device_marked(const std::atomic<uint64_t>& done, int dev) { return (done.load(std::memory_order_acquire) >> dev) & 1u; }
+inline void mark_device(std::atomic<uint64_t>& done, int dev) { done.fetch_or(1ull << dev, std::memory_order_release); }
 
 inline tdq_status cuda_status(cudaError_t e) { return e == cudaSuccess ? TDQ_OK : TDQ_ERR_CUDA; }
 

@@ -847,15 +847,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
 
 using namespace tdq;
 
-static int sm_count() {
-    static int n_sm = 0;
-    if (n_sm == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return 0;
-        if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n_sm = 0;
-    }
-    return n_sm;
-}
+static int sm_count() { return current_device_sm_count(); }
 
 extern "C" size_t tdq_linear_workspace_bytes(int64_t M, int64_t I_pad, int64_t O, int32_t group_size) {
     if (M < 0 || I_pad <= 0 || O <= 0 || group_size <= 0 || group_size % 32 || I_pad % group_size)
@@ -866,6 +858,17 @@ extern "C" size_t tdq_linear_workspace_bytes(int64_t M, int64_t I_pad, int64_t O
 }
 
 namespace tdq {
+
+tdq_status linear_check_shape(int64_t M, int64_t I_pad, int64_t O, int32_t group_size, size_t workspace_bytes) {
+    if (M < 0 || O <= 0 || I_pad <= 0) return TDQ_ERR_INVALID_ARG;
+    if (group_size <= 0 || I_pad % group_size) return TDQ_ERR_INVALID_ARG;
+    if (group_size % 32 || group_size > 4096) return TDQ_ERR_UNSUPPORTED;
+    if (I_pad / 2 > INT32_MAX) return TDQ_ERR_INVALID_ARG;
+    Plan p;
+    if (!make_plan(M, I_pad, O, group_size, 148, p)) return TDQ_ERR_UNSUPPORTED;
+    if (workspace_bytes < kWorkspaceHeader + p.a_bytes + p.b_bytes + p.s_bytes) return TDQ_ERR_WORKSPACE;
+    return TDQ_OK;
+}
 
 tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* xscale, const uint8_t* wcodes,
                        const float* wscale, const float* bias, int64_t M, int64_t I_pad, int64_t O, int32_t group_size,
@@ -1030,6 +1033,40 @@ extern "C" tdq_status tdq_workspace_status(const void* workspace, void* cuda_str
 }
 
 // ------------------------------------------------------------------------------------------
+// tdq_selftest_wait_timeout: makes a bounded wait run out, the way a lost arrival would
+
+namespace tdq {
+namespace {
+// One warp: a fresh barrier with one expected arrival that never comes, waited on with the GEMM kernels' own
+// routine and a short limit; the code lands in the workspace's status word.  Nothing is in flight when the
+// warp leaves.
+__global__ void __launch_bounds__(32) linear_wait_selftest_kernel(uint32_t* status, long long limit) {
+    __shared__ Ctrl c;
+    if (threadIdx.x == 0) {
+        mbar_init(&c.full[0], 1);
+        c.abort_flag = 0;
+    }
+    __syncwarp();
+    mbar_wait_warp(&c.full[0], 0u, &c, status, 15u, limit);
+}
+}  // namespace
+}  // namespace tdq
+
+extern "C" tdq_status tdq_selftest_wait_timeout(int32_t which, int64_t limit_cycles, void* workspace, void* cuda_stream) {
+    if (which != 0 && which != 1) return TDQ_ERR_INVALID_ARG;
+    if (limit_cycles < 1000 || limit_cycles > 2000000000LL) return TDQ_ERR_INVALID_ARG;   // at most about a second
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    if (which == 1) return act_wait_selftest(limit_cycles, stream);
+    if (!workspace) return TDQ_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(workspace) % 16) return TDQ_ERR_ALIGNMENT;
+    if (cudaMemsetAsync(workspace, 0, 16, stream) != cudaSuccess) return TDQ_ERR_CUDA;
+    linear_wait_selftest_kernel<<<1, 32, 0, stream>>>(reinterpret_cast<uint32_t*>(workspace), limit_cycles);
+    if (cudaGetLastError() != cudaSuccess) return TDQ_ERR_CUDA;
+    g_launch_count.fetch_add(1, std::memory_order_relaxed);
+    return TDQ_OK;
+}
+
+// ------------------------------------------------------------------------------------------
 // tdq_w4a4_linear_static: the same two kernels, with the operand blocks in a fixed device array
 
 namespace {
@@ -1038,7 +1075,6 @@ constexpr size_t kStaticScratchBytes = TDQ_LINEAR_STATIC_BYTES;
 // use the name to look its device address up; the kernels get that address as a plain pointer.
 static __device__ __align__(256) uint8_t g_static_scratch[kStaticScratchBytes];
 
-constexpr int kMaxDevices = 64;
 std::mutex g_static_mutex;
 void* g_static_ptr[kMaxDevices] = {};
 }  // namespace

@@ -209,6 +209,9 @@ __global__ void __launch_bounds__(kFastThreads) act_g32_kernel(ActArgs a) {
 constexpr int kRingStagesBf16 = 4, kRingStagesF32 = 3;
 constexpr int kRingThreads = kFastThreads + 32;
 constexpr long long kRingTimeout = 2000000000LL;
+// A ring wait that ran out leaves its code here (first writer wins): bits 0-7 name the wait (12 producer, 13 consumer,
+// 14 the self-test), bits 8-31 the CTA.  One word per device, read and cleared by tdq_quantize_status().
+__device__ uint32_t g_act_wait_status = 0u;
 
 __device__ __forceinline__ uint32_t ring_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ bool ring_test(uint64_t* bar, uint32_t parity) {
@@ -223,7 +226,8 @@ __device__ __forceinline__ bool ring_test(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 // false when the phase did not complete in about a second (the caller then stops working)
-__device__ __forceinline__ bool ring_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool ring_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, uint32_t code,
+                                          long long limit = kRingTimeout) {
     if (ring_test(bar, parity)) return true;
     long long t0 = 0;
     uint32_t polls = 0;
@@ -233,7 +237,11 @@ __device__ __forceinline__ bool ring_wait(uint64_t* bar, uint32_t parity, volati
             if (*abort_flag) return false;
             const long long now = clock64();
             if (t0 == 0) t0 = now;
-            if (now - t0 > kRingTimeout) { *abort_flag = 1; return false; }
+            if (now - t0 > limit) {
+                atomicCAS(&g_act_wait_status, 0u, code | ((uint32_t)blockIdx.x << 8));
+                *abort_flag = 1;
+                return false;
+            }
         }
     }
     return true;
@@ -263,7 +271,7 @@ __global__ void __launch_bounds__(kRingThreads) act_g32_ring_kernel(ActArgs a, i
         if (t == kFastThreads) {   // producer lane
             uint32_t s = 0, ph = 0;
             for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
-                if (!ring_wait(&empty[s], ph ^ 1, &abort_flag)) break;
+                if (!ring_wait(&empty[s], ph ^ 1, &abort_flag, 12u)) break;
                 const int64_t g0 = tile * kFastThreads;
                 const int64_t ng = min((int64_t)kFastThreads, a.total_groups - g0);
                 const uint32_t bytes = (uint32_t)(ng * kGroupBytes);
@@ -279,7 +287,7 @@ __global__ void __launch_bounds__(kRingThreads) act_g32_ring_kernel(ActArgs a, i
     }
     uint32_t s = 0, ph = 0;
     for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
-        if (!__all_sync(0xffffffffu, ring_wait(&full[s], ph, &abort_flag))) break;
+        if (!__all_sync(0xffffffffu, ring_wait(&full[s], ph, &abort_flag, 13u))) break;
         const int64_t gi = tile * kFastThreads + t;
         uint32_t w[kChunks * 4];
         // volatile loads: the stage is handed back right below, so these must be the only reads of it
@@ -306,17 +314,14 @@ template <bool BF16, int KZR, int KB = 32>
 cudaError_t launch_ring(const ActArgs& a, cudaStream_t st) {
     constexpr int kStages = BF16 ? kRingStagesBf16 : kRingStagesF32;
     constexpr int smem = kStages * kFastThreads * (BF16 ? 64 : 128);
-    static int n_sm = 0;
-    static bool attr_done = false;
-    if (n_sm == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorUnknown;
-        if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return cudaErrorUnknown;
-    }
-    if (!attr_done) {
+    static std::atomic<uint64_t> attr_done{0};      // per template instance, one bit per device
+    int dev = 0;
+    const int n_sm = current_device_sm_count(&dev);
+    if (n_sm <= 0) return cudaErrorUnknown;
+    if (!device_marked(attr_done, dev)) {
         cudaError_t e = cudaFuncSetAttribute(act_g32_ring_kernel<BF16, KZR, KB>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
-        attr_done = true;
+        mark_device(attr_done, dev);
     }
     const int64_t n_tiles = (a.total_groups + kFastThreads - 1) / kFastThreads;
     const int64_t grid = n_tiles < 2 * n_sm ? n_tiles : 2 * n_sm;
@@ -673,4 +678,46 @@ extern "C" tdq_status tdq_quantize_act_fixed(const void* x, tdq_dtype x_dtype, i
     if (cudaGetLastError() != cudaSuccess) return TDQ_ERR_CUDA;
     g_launch_count.fetch_add(1, std::memory_order_relaxed);
     return TDQ_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// bounded waits of the quantizer: the status word and the self-test
+
+namespace tdq {
+namespace {
+// One warp: a fresh barrier with one expected arrival that never comes, waited on with the ring kernel's own
+// routine and a short limit.  Nothing is in flight when the warp leaves.
+__global__ void __launch_bounds__(32) act_wait_selftest_kernel(long long limit) {
+    __shared__ uint64_t bar;
+    __shared__ volatile int abort_flag;
+    if (threadIdx.x == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(ring_smem_u32(&bar)) : "memory");
+        abort_flag = 0;
+    }
+    __syncwarp();
+    ring_wait(&bar, 0u, &abort_flag, 14u, limit);
+}
+}  // namespace
+
+tdq_status act_wait_selftest(long long limit_cycles, cudaStream_t stream) {
+    act_wait_selftest_kernel<<<1, 32, 0, stream>>>(limit_cycles);
+    if (cudaGetLastError() != cudaSuccess) return TDQ_ERR_CUDA;
+    g_launch_count.fetch_add(1, std::memory_order_relaxed);
+    return TDQ_OK;
+}
+}  // namespace tdq
+
+extern "C" tdq_status tdq_quantize_status(void* cuda_stream, uint32_t* detail) {
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    uint32_t word = 0;
+    const uint32_t zero = 0;
+    if (cudaMemcpyFromSymbolAsync(&word, g_act_wait_status, sizeof word, 0, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return TDQ_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return TDQ_ERR_CUDA;
+    if (word != 0 &&
+        (cudaMemcpyToSymbolAsync(g_act_wait_status, &zero, sizeof zero, 0, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+         cudaStreamSynchronize(stream) != cudaSuccess))
+        return TDQ_ERR_CUDA;
+    if (detail) *detail = word;
+    return word == 0 ? TDQ_OK : TDQ_ERR_DEVICE_TIMEOUT;
 }

@@ -139,7 +139,8 @@ __device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
 // Slow path of a bounded wait: sleeps on the barrier until the phase completes, another role of
 // this CTA has given up, or about a second has passed; then it records which wait gave up
 // (first writer wins) and raises the CTA-wide flag.
-__device__ __forceinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, Ctrl* c, uint32_t* status, uint32_t code) {
+__device__ __forceinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, Ctrl* c, uint32_t* status, uint32_t code,
+                                               long long limit = kTimeoutCycles) {
     long long t0 = 0;
 #pragma unroll 1
     for (;;) {
@@ -151,7 +152,7 @@ __device__ __forceinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, C
         if (c->abort_flag) return false;
         const long long now = clock64();
         if (t0 == 0) t0 = now;
-        if (now - t0 > kTimeoutCycles) {
+        if (now - t0 > limit) {
             atomicCAS(status, 0u, code | ((uint32_t)blockIdx.x << 8));
             c->abort_flag = 1;
             return false;
@@ -160,9 +161,10 @@ __device__ __forceinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, C
 }
 
 // Bounded wait by a converged warp; the answer is the same in every lane.
-__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, Ctrl* c, uint32_t* status, uint32_t code) {
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, Ctrl* c, uint32_t* status, uint32_t code,
+                                               long long limit = kTimeoutCycles) {
     if (__all_sync(0xffffffffu, mbar_test(bar, parity))) return true;
-    return __all_sync(0xffffffffu, mbar_wait_slow(bar, parity, c, status, code));
+    return __all_sync(0xffffffffu, mbar_wait_slow(bar, parity, c, status, code, limit));
 }
 
 // The same primitives on 32-bit shared-window addresses, for the hot loops (no pointer conversion).

@@ -83,3 +83,45 @@ def test_binding_refuses_cpu_tensors(tdq):
     import torch
     with pytest.raises(ValueError):
         tdq.quantize_act(torch.zeros(4, 64))
+
+
+@pytest.mark.gpu
+def test_binding_refuses_layouts_the_abi_cannot_see(tdq):
+    """dtype, contiguity and column pitch are checked before any pointer reaches the library (no launch)."""
+    import torch
+    n0 = tdq.kernel_launch_count()
+    xc = torch.zeros((8, 32), dtype=torch.uint8, device="cuda")
+    xs = torch.ones((8, 2), device="cuda")
+    wc = torch.zeros((16, 32), dtype=torch.uint8, device="cuda")
+    ws = torch.ones((16,), device="cuda")
+    with pytest.raises(TypeError):
+        tdq.w4a4_linear(xc, xs.double(), wc, ws)
+    with pytest.raises(TypeError):
+        tdq.w4a4_linear(xc.to(torch.int8), xs, wc, ws)
+    with pytest.raises(ValueError):
+        tdq.w4a4_linear(xc, xs, wc.t().contiguous().t(), ws)                 # transposed view
+    with pytest.raises(ValueError):
+        tdq.w4a4_linear(xc, xs, wc, ws, y=torch.zeros((16, 8), device="cuda").t())   # columns not adjacent
+    with pytest.raises(ValueError):
+        tdq.w4a4_linear(xc, xs, wc, torch.ones((32,), device="cuda")[::2])
+    assert tdq.kernel_launch_count() == n0
+
+
+def test_wait_selftest_and_host_call_argument_checks(tdq):
+    L = tdq.lib()
+    fake = ctypes.c_void_p(0x1000)
+    n0 = tdq.kernel_launch_count()
+    assert L.tdq_selftest_wait_timeout(2, 100000, fake, None) == tdq.ERR_INVALID_ARG
+    assert L.tdq_selftest_wait_timeout(0, 10, fake, None) == tdq.ERR_INVALID_ARG
+    assert L.tdq_selftest_wait_timeout(0, 1 << 40, fake, None) == tdq.ERR_INVALID_ARG
+    assert L.tdq_selftest_wait_timeout(0, 100000, None, None) == tdq.ERR_INVALID_ARG
+    assert L.tdq_selftest_wait_timeout(0, 100000, ctypes.c_void_p(0x1004), None) == tdq.ERR_ALIGNMENT
+    # the host-buffer call refuses what either of its two calls would refuse, before it queues anything
+    p = tdq.default_act_params()
+    host = lambda pp, ws_bytes, O=64, C=64: L.tdq_quant_linear_host(fake, 1, 1, 256, C, ctypes.byref(pp), fake, fake, None, O,
+                                                                   fake, 0, fake, fake, fake, fake, fake, ws_bytes, None)
+    assert host(tdq.act_params(g=16), 1 << 24) == tdq.ERR_UNSUPPORTED          # the linear layer wants g % 32 == 0
+    assert host(tdq.act_params(tau=0.0), 1 << 24) == tdq.ERR_INVALID_ARG
+    assert host(p, 64) == tdq.ERR_WORKSPACE
+    assert host(p, 1 << 24, O=0) == tdq.ERR_INVALID_ARG
+    assert tdq.kernel_launch_count() == n0
