@@ -79,10 +79,11 @@ void tdq_default_act_params(tdq_act_params* p /* HOST, out */);
  *
  *   x          [B*N rows, C] row-major, x_dtype, consecutive rows row_stride_elems apart
  *              (>= C).  No alignment is required; 16-byte aligned x with C % 32 == 0,
- *              row_stride_elems % 8 == 0 and g == 32 takes the fast kernel (any zero-bin rank
- *              with the maximum as base radius; base ranks 29-31 with zero-bin rank 7 or
- *              TDQ_ENABLE_C2 off; anything else takes a much slower general kernel with the
- *              same results).
+ *              row_stride_elems % 8 == 0 and g == 32 takes the fast kernels, whatever the two
+ *              ranks (the maximum as base radius with any zero-bin rank, and base ranks 29-31
+ *              with zero-bin rank 7, have kernels of their own; any other pair runs a kernel
+ *              that takes its ranks at run time, about a fifth slower); anything else takes a
+ *              much slower general kernel with the same results.
  *   codes      [B*N, C_pad/2] bytes; byte j of a row holds channel 2j in its low nibble
  *              and channel 2j+1 in its high nibble, two's complement.
  *   scale      [B*N, K] float32, Delta_k.
@@ -137,6 +138,19 @@ tdq_status tdq_quantize_act_fixed(const void* x, tdq_dtype x_dtype, int64_t B, i
  */
 tdq_status tdq_quantize_weight(const void* w, tdq_dtype w_dtype, int64_t O, int64_t I, int32_t pad_to,
                                uint8_t* wcodes, float* wscale, void* cuda_stream);
+
+/*
+ * The affine mode of the auxiliary Linear I/O correction of Supp. S1.1 (modes none / bias / affine; the paper
+ * names the modes without a formula, the reading taken here is a per-output-channel y' = a_o y + b_o applied to
+ * the layer's output y = s_o Sigma + bias_o).  The correction is static, so it costs nothing at run time when it
+ * is folded into the layer's constants once:  wscale_out[o] = a_o s_o,  bias_out[o] = a_o bias_o + b_o, each
+ * rounded to binary32; tdq_w4a4_linear (or the fused call) with these two vectors then computes y'.  The result
+ * differs from a_o (s_o Sigma + bias_o) + b_o evaluated exactly by a few units in the last place of its terms.
+ *   wscale [O], bias NULL or [O], out_mul [O] (a_o), out_add NULL or [O] (b_o); wscale_out [O] and bias_out [O]
+ *   may alias wscale and bias.  The bias mode of the correction is the bias vector of tdq_w4a4_linear itself.
+ */
+tdq_status tdq_fold_output_affine(const float* wscale, const float* bias, const float* out_mul, const float* out_add,
+                                  int64_t O, float* wscale_out, float* bias_out, void* cuda_stream);
 
 /*
  * W4A4 linear layer, Algorithm S1 step 10 with x_hat = Delta_k q (Eq. 9) and

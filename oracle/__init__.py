@@ -179,3 +179,18 @@ def w4a4_linear(xcodes, xscale, wcodes, wscale, bias=None, g=32, want_acc=False)
     if want_acc:
         out["acc"] = acc
     return out
+
+
+def output_affine(ref, out_mul, out_add=None, bias=None):
+    """The affine mode of the auxiliary Linear I/O correction (Supp. S1.1): y' = a_o * y + b_o per output channel,
+    applied in binary64 to the dict w4a4_linear returns (y_d, t_abs; y is y_d rounded to binary32).  t_abs, the
+    diagnostic size of the summed terms, is scaled by |a_o|; when the layer's bias is passed, |a_o bias_o| and
+    |b_o| are added to it (the constants a folded evaluation rounds)."""
+    a = np.asarray(out_mul, np.float64)[None, :]
+    b = 0.0 if out_add is None else np.asarray(out_add, np.float64)[None, :]
+    y_d = a * ref["y_d"] + b
+    t_abs = np.abs(a) * ref["t_abs"]
+    if bias is not None:
+        t_abs = t_abs + np.abs(a * np.asarray(bias, np.float64)[None, :])
+        t_abs = t_abs + np.abs(b)
+    return dict(y=y_d.astype(np.float32), y_d=y_d, t_abs=t_abs)

@@ -24,7 +24,7 @@ ENABLE_C1, ENABLE_C2, POW2_STEP = 1, 2, 4
 EXPORTS = ["tdq_default_act_params", "tdq_quantize_act", "tdq_quantize_weight", "tdq_w4a4_linear",
            "tdq_quant_linear_fused", "tdq_quant_linear_host", "tdq_quantize_act_nchw", "tdq_quantize_act_fixed", "tdq_w4a4_linear_pow2", "tdq_linear_workspace_bytes",
            "tdq_workspace_status", "tdq_status_string", "tdq_kernel_launch_count", "tdq_w4a4_linear_static",
-           "tdq_quantize_status", "tdq_selftest_wait_timeout"]
+           "tdq_quantize_status", "tdq_selftest_wait_timeout", "tdq_fold_output_affine"]
 
 
 class ActParams(ctypes.Structure):
@@ -66,6 +66,8 @@ _lib.tdq_quantize_status.argtypes = [_vp, ctypes.POINTER(ctypes.c_uint32)]
 _lib.tdq_quantize_status.restype = ctypes.c_int
 _lib.tdq_selftest_wait_timeout.argtypes = [_i32, _i64, _vp, _vp]
 _lib.tdq_selftest_wait_timeout.restype = ctypes.c_int
+_lib.tdq_fold_output_affine.argtypes = [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _vp]
+_lib.tdq_fold_output_affine.restype = ctypes.c_int
 _lib.tdq_status_string.argtypes = [ctypes.c_int]
 _lib.tdq_status_string.restype = ctypes.c_char_p
 _lib.tdq_kernel_launch_count.argtypes = []
@@ -363,3 +365,16 @@ def selftest_wait_timeout(which: int, limit_cycles: int, workspace: torch.Tensor
     dev = workspace.device if workspace is not None else None
     _check(_lib.tdq_selftest_wait_timeout(which, limit_cycles, ws, ctypes.c_void_p(torch.cuda.current_stream(dev).cuda_stream)),
            "tdq_selftest_wait_timeout")
+
+
+def fold_output_affine(wscale, bias, out_mul, out_add=None):
+    """tdq_fold_output_affine: (wscale', bias') such that the linear layer computes out_mul * y + out_add."""
+    _need_cuda(wscale, bias, out_mul, out_add)
+    dev = _check_operands([("wscale", wscale, torch.float32), ("bias", bias, torch.float32), ("out_mul", out_mul, torch.float32),
+                           ("out_add", out_add, torch.float32)])
+    O = wscale.shape[0]
+    ws2, b2 = torch.empty_like(wscale), torch.empty_like(wscale)
+    with torch.cuda.device(dev):
+        _check(_lib.tdq_fold_output_affine(_ptr(wscale), _ptr(bias), _ptr(out_mul), _ptr(out_add), O, _ptr(ws2), _ptr(b2),
+                                           _stream(wscale)), "tdq_fold_output_affine")
+    return ws2, b2

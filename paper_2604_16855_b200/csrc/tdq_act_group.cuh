@@ -136,13 +136,37 @@ __device__ __forceinline__ float kth_of_sorted_halves_f32(const float (&s)[32]) 
     return r;
 }
 
+// The same with the rank known only at run time: a switch over the 32 compile-time instances, so that the sorted
+// halves are only ever indexed with constants and stay in registers.
+#define TDQ_RANK_CASES \
+    TDQ_RC(1) TDQ_RC(2) TDQ_RC(3) TDQ_RC(4) TDQ_RC(5) TDQ_RC(6) TDQ_RC(7) TDQ_RC(8) TDQ_RC(9) TDQ_RC(10) TDQ_RC(11) \
+    TDQ_RC(12) TDQ_RC(13) TDQ_RC(14) TDQ_RC(15) TDQ_RC(16) TDQ_RC(17) TDQ_RC(18) TDQ_RC(19) TDQ_RC(20) TDQ_RC(21) \
+    TDQ_RC(22) TDQ_RC(23) TDQ_RC(24) TDQ_RC(25) TDQ_RC(26) TDQ_RC(27) TDQ_RC(28) TDQ_RC(29) TDQ_RC(30) TDQ_RC(31) TDQ_RC(32)
+__device__ __forceinline__ uint32_t kth_of_sorted_halves_u16_rt(const uint32_t (&s)[16], int k) {
+    switch (k) {
+#define TDQ_RC(K_) case K_: return kth_of_sorted_halves_u16<K_>(s);
+        TDQ_RANK_CASES
+#undef TDQ_RC
+    }
+    return 0u;
+}
+__device__ __forceinline__ float kth_of_sorted_halves_f32_rt(const float (&s)[32], int k) {
+    switch (k) {
+#define TDQ_RC(K_) case K_: return kth_of_sorted_halves_f32<K_>(s);
+        TDQ_RANK_CASES
+#undef TDQ_RC
+    }
+    return 0.0f;
+}
+
 // One group held in registers (w: 16 packed bf16 pairs or 32 floats, in channel order): statistics,
 // projection, quantization.  out: the group's 32 two's complement nibbles, channel 8 w + n in
 // nibble n of word w; delta: its step.  KB: rank of the base radius among the magnitudes (32: the maximum,
 // Eq. 5; less: the percentile option of Supp. S4.8, which takes the group's KB-th smallest magnitude).
+// KB == 0: both ranks are run-time values (rt_kzr, rt_kb in 1..32), for the settings that have no instance of their own.
 template <bool BF16, int KZR, int KB = 32>
 __device__ __forceinline__ void quantize_group32(const uint32_t (&w)[BF16 ? 16 : 32], float seven_tau, uint32_t flags,
-                                                 uint32_t (&out)[4], float& delta) {
+                                                 uint32_t (&out)[4], float& delta, int rt_kzr = 0, int rt_kb = 0) {
     auto get = [&](int i) -> float {
         if (BF16) return (i & 1) ? __uint_as_float(w[i >> 1] & 0xffff0000u) : __uint_as_float(w[i >> 1] << 16);
         return __uint_as_float(w[i]);
@@ -159,8 +183,13 @@ __device__ __forceinline__ void quantize_group32(const uint32_t (&w)[BF16 ? 16 :
 #define TDQ_CE(i, j) { uint32_t lo_ = __vminu2(s[i], s[j]); s[j] = __vmaxu2(s[i], s[j]); s[i] = lo_; }
 #include "sort16_network.inc"
 #undef TDQ_CE
-            c_base = __uint_as_float(kth_of_sorted_halves_u16<KB>(s) << 16);
-            if (flags & TDQ_ENABLE_C2) thr = __uint_as_float(kth_of_sorted_halves_u16<KZR>(s) << 16);
+            if (KB == 0) {
+                c_base = __uint_as_float(kth_of_sorted_halves_u16_rt(s, rt_kb) << 16);
+                if (flags & TDQ_ENABLE_C2) thr = __uint_as_float(kth_of_sorted_halves_u16_rt(s, rt_kzr) << 16);
+            } else {
+                c_base = __uint_as_float(kth_of_sorted_halves_u16<(KB ? KB : 1)>(s) << 16);
+                if (flags & TDQ_ENABLE_C2) thr = __uint_as_float(kth_of_sorted_halves_u16<(KZR ? KZR : 1)>(s) << 16);
+            }
         } else {
             float s[32];
 #pragma unroll
@@ -171,8 +200,13 @@ __device__ __forceinline__ void quantize_group32(const uint32_t (&w)[BF16 ? 16 :
 #define TDQ_CE(i, j) { float lo_ = fminf(s[16 + i], s[16 + j]); s[16 + j] = fmaxf(s[16 + i], s[16 + j]); s[16 + i] = lo_; }
 #include "sort16_network.inc"
 #undef TDQ_CE
-            c_base = kth_of_sorted_halves_f32<KB>(s);
-            if (flags & TDQ_ENABLE_C2) thr = kth_of_sorted_halves_f32<KZR>(s);
+            if (KB == 0) {
+                c_base = kth_of_sorted_halves_f32_rt(s, rt_kb);
+                if (flags & TDQ_ENABLE_C2) thr = kth_of_sorted_halves_f32_rt(s, rt_kzr);
+            } else {
+                c_base = kth_of_sorted_halves_f32<(KB ? KB : 1)>(s);
+                if (flags & TDQ_ENABLE_C2) thr = kth_of_sorted_halves_f32<(KZR ? KZR : 1)>(s);
+            }
         }
     } else if (BF16) {
         // |x| of a bf16 is a 15-bit key whose unsigned order is the numeric order, so the network

@@ -139,7 +139,7 @@ template <bool BF16, int KZR, int KB = 32>
 __device__ __forceinline__ void process_group(const uint32_t (&w)[BF16 ? 16 : 32], const ActArgs& a, int64_t gi) {
     uint32_t out[4];
     float delta;
-    quantize_group32<BF16, KZR, KB>(w, a.seven_tau, a.flags, out, delta);
+    quantize_group32<BF16, KZR, KB>(w, a.seven_tau, a.flags, out, delta, a.k_zr, a.k_base);
     reinterpret_cast<uint4*>(a.codes)[gi] = make_uint4(out[0], out[1], out[2], out[3]);
     a.scale[gi] = delta;
     if (a.offset) a.offset[gi] = 0.0f;
@@ -339,8 +339,13 @@ template <bool BF16>
 cudaError_t launch_fast(const ActArgs& a, cudaStream_t st) {
     const int64_t blocks = (a.total_groups + kFastThreads - 1) / kFastThreads;
     dim3 grid((unsigned)blocks), block(kFastThreads);
+    if (a.k_base != 32 && (a.k_base < 29 || a.k_zr != 7)) {
+        // any other pair of ranks: the instance that takes both at run time
+        if (a.row_stride == a.C) return launch_ring<BF16, 0, 0>(a, st);
+        act_g32_kernel<BF16, 0, 0><<<grid, block, 0, st>>>(a);
+        return cudaGetLastError();
+    }
     if (a.k_base != 32) {        // percentile base radius: ranks 29..31 beside the default zero-bin rank
-        if (a.k_zr != 7) return cudaErrorInvalidValue;
         switch (a.k_base) {
 #define TDQ_CASE(KB_)                                                                  \
             case KB_:                                                                  \
@@ -514,12 +519,9 @@ __global__ void __launch_bounds__(256) act_fixed_kernel(FixedArgs f) {
 
 // the zero-bin ranks the channel-major kernel is instantiated for (those of the paper's sweep over zr)
 bool fast_rank(int k) { return k == 4 || k == 7 || k == 10 || k == 13 || k == 16 || k == 32; }
-// base radius: the maximum, or one of the three ranks below it together with the default zero-bin rank
-bool fast_base_rank(const tdq_act_params* p) {
-    const int kb = rank_of(p->base_percentile, 32);
-    if (kb == 32) return true;
-    return kb >= 29 && (!(p->flags & TDQ_ENABLE_C2) || rank_of(p->zr, 32) == 7);
-}
+// base radius: any rank (the maximum and ranks 29-31 with the default zero-bin rank have instances of their own, the
+// other pairs share the instance that takes its ranks at run time)
+bool fast_base_rank(const tdq_act_params*) { return true; }
 
 }  // namespace
 

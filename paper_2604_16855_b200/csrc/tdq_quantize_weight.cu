@@ -50,6 +50,17 @@ __global__ void __launch_bounds__(kWThreads) weight_quant_kernel(const void* w, 
     }
 }
 
+// The affine output correction folded into the layer's constants: a (s Sigma + bias) + b = (a s) Sigma + (a bias + b).
+__global__ void fold_affine_kernel(const float* wscale, const float* bias, const float* mul, const float* add, int64_t O,
+                                   float* wscale_out, float* bias_out) {
+    const int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (o >= O) return;
+    const float a = mul[o];
+    wscale_out[o] = __fmul_rn(a, wscale[o]);
+    const float ab = bias ? __fmul_rn(a, bias[o]) : 0.0f;
+    bias_out[o] = add ? __fadd_rn(ab, add[o]) : ab;
+}
+
 }  // namespace
 }  // namespace tdq
 
@@ -67,6 +78,18 @@ extern "C" tdq_status tdq_quantize_weight(const void* w, tdq_dtype w_dtype, int6
         weight_quant_kernel<true><<<(unsigned)O, kWThreads, 0, stream>>>(w, I, I_pad, wcodes, wscale);
     else
         weight_quant_kernel<false><<<(unsigned)O, kWThreads, 0, stream>>>(w, I, I_pad, wcodes, wscale);
+    if (cudaGetLastError() != cudaSuccess) return TDQ_ERR_CUDA;
+    g_launch_count.fetch_add(1, std::memory_order_relaxed);
+    return TDQ_OK;
+}
+
+extern "C" tdq_status tdq_fold_output_affine(const float* wscale, const float* bias, const float* out_mul, const float* out_add,
+                                             int64_t O, float* wscale_out, float* bias_out, void* cuda_stream) {
+    if (!wscale || !out_mul || !wscale_out || !bias_out) return TDQ_ERR_INVALID_ARG;
+    if (O < 0 || O > INT32_MAX) return TDQ_ERR_INVALID_ARG;
+    if (O == 0) return TDQ_OK;
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    fold_affine_kernel<<<(unsigned)((O + 255) / 256), 256, 0, stream>>>(wscale, bias, out_mul, out_add, O, wscale_out, bias_out);
     if (cudaGetLastError() != cudaSuccess) return TDQ_ERR_CUDA;
     g_launch_count.fetch_add(1, std::memory_order_relaxed);
     return TDQ_OK;

@@ -214,3 +214,54 @@ def test_row_shards_equal_the_unsharded_call(tdq, idx, rows, split):
         yf0 = tdq.quant_linear_fused(xt[:split], wc, ws, bias)
         yf1 = tdq.quant_linear_fused(xt[split:].contiguous(), wc, ws, bias)
         assert torch.equal(torch.cat([yf0, yf1]).view(torch.int32), y_all.view(torch.int32))
+
+
+# ---------------------------------------------------------------------------------------
+# percentile base radius at any rank, with any zero-bin rank, on the fast kernels (ranks taken at run time)
+
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("p,zr,flags", [(0.5, 0.2, 3), (0.75, 0.2, 3), (0.25, 0.1, 3), (0.04, 0.2, 3), (0.85, 0.5, 3), (0.6, 1.0, 3),
+                                        (0.95, 0.4, 3), (0.7, 0.2, 1), (0.3, 0.3, 2), (0.5, 0.2, 0), (0.999, 0.03, 3)])
+def test_any_pair_of_ranks_on_the_fast_kernels(tdq, bf16, p, zr, flags):
+    n0 = None
+    for x, stride_pad in ((si.config3().x.reshape(-1, 320)[:2000], 0), (si.edge_rows(C=64), 0), (si.dc_offset_tokens(M=700, C=96), 32)):
+        if x.dtype == np.uint16:
+            x = si.bf16_bits_to_f32(x)
+        xin = si.f32_to_bf16_bits(x) if bf16 else x
+        ref = oracle.quantize_act(xin, p=p, zr=zr, flags=flags)
+        xt = to_cuda(xin, bf16=bf16)
+        if stride_pad:                                # rows with a pitch: the strided fast kernel
+            wide = torch.zeros((xt.shape[0], xt.shape[1] + stride_pad), dtype=xt.dtype, device="cuda")
+            wide[:, : xt.shape[1]] = xt
+            xt = wide[:, : x.shape[1]]
+        codes, scale = tdq.quantize_act(xt, tdq.act_params(p=p, zr=zr, flags=flags))
+        torch.cuda.synchronize()
+        rep = compare_quantizer(_f32(xin, bf16), 32, ref, codes.cpu().numpy(), scale.cpu().numpy())
+        assert rep["code_mismatch"] == 0 and rep["scale_exact_frac"] == 1.0, rep
+
+
+# ---------------------------------------------------------------------------------------
+# the affine output correction, folded into the layer's constants
+
+@pytest.mark.parametrize("with_bias,with_shift,fused", [(True, True, False), (False, True, False), (True, False, True), (False, False, False)])
+def test_affine_output_correction_folded_into_the_constants(tdq, with_bias, with_shift, fused):
+    case = si.config3()
+    x = case.x.reshape(-1, case.C)[:1300]
+    rng = np.random.default_rng(17)
+    O = case.O
+    bias = rng.standard_normal(O).astype(np.float32) * 0.05 if with_bias else None
+    a = (rng.uniform(0.5, 1.5, O) * rng.choice([-1.0, 1.0], O)).astype(np.float32)
+    b = rng.standard_normal(O).astype(np.float32) * 0.1 if with_shift else None
+    xt = to_cuda(x, bf16=True)
+    wc, ws = tdq.quantize_weight(to_cuda(case.w))
+    ws2, b2 = tdq.fold_output_affine(ws, None if bias is None else to_cuda(bias), to_cuda(a), None if b is None else to_cuda(b))
+    if fused:
+        y = tdq.quant_linear_fused(xt, wc, ws2, b2)
+    else:
+        codes, scale = tdq.quantize_act(xt)
+        y = tdq.w4a4_linear(codes, scale, wc, ws2, b2)
+    xa, wq = oracle.quantize_act(x), oracle.quantize_weight(case.w)
+    ref = oracle.output_affine(oracle.w4a4_linear(xa["codes"], xa["scale"], wq["codes"], wq["scale"], bias=bias), a, b,
+                               bias=np.zeros(O, np.float32) if bias is None else bias)
+    # three more roundings than the plain layer (a_o s_o, a_o bias_o, + b_o), counted against the size of the terms
+    compare_y(y.cpu().numpy(), ref, case.C // 32 + 3)

@@ -319,6 +319,34 @@ def test_linear_equals_float64_product_of_dequantized_operands(C, O, g):
     np.testing.assert_allclose(nb["y_d"], want - bias, rtol=0, atol=float(1e-12 * scale_ref.max()))
 
 
+def test_output_affine_is_a_diagonal_layer_after_the_linear_layer():
+    """The affine correction (Supp. S1.1): against a float64 product with a diagonal matrix appended; the identity
+    and pure-shift special cases; a swapped multiplier and shift, or a per-row instead of per-column vector, fail."""
+    rng = np.random.default_rng(5)
+    C, O = 96, 40
+    x = si.token_mixture(rng, 1, 30, C, sigma_log_std=0.5, bg_frac=0.1, bg_nu=3.0, bg_amp=20.0).reshape(-1, C)
+    w = si.weights(rng, O, C)
+    bias = rng.standard_normal(O).astype(np.float32)
+    a = rng.uniform(0.5, 1.5, O).astype(np.float32) * rng.choice([-1.0, 1.0], O).astype(np.float32)
+    b = rng.standard_normal(O).astype(np.float32)
+    xa, wq = oracle.quantize_act(x), oracle.quantize_weight(w)
+    ref = oracle.w4a4_linear(xa["codes"], xa["scale"], wq["codes"], wq["scale"], bias=bias)
+    out = oracle.output_affine(ref, a, b)
+    K = xa["scale"].shape[1]
+    x_hat = (xa["q"].reshape(-1, K, 32) * xa["scale"].astype(np.float64)[..., None]).reshape(-1, K * 32)
+    w_hat = wq["q"] * wq["scale"].astype(np.float64)[:, None]
+    want = (x_hat @ w_hat.T + bias.astype(np.float64)) @ np.diag(a.astype(np.float64)) + b.astype(np.float64)
+    size = (np.abs(x_hat) @ np.abs(w_hat).T + np.abs(bias)) * np.abs(a) + np.abs(b)
+    assert (np.abs(out["y_d"] - want) <= 1e-12 * size).all()
+    np.testing.assert_array_equal(out["y"], out["y_d"].astype(np.float32))
+    np.testing.assert_allclose(out["t_abs"], np.abs(a.astype(np.float64)) * ref["t_abs"], rtol=1e-15)
+    same = oracle.output_affine(ref, np.ones(O, np.float32))
+    np.testing.assert_array_equal(same["y_d"], ref["y_d"])
+    shift = oracle.output_affine(ref, np.ones(O, np.float32), b)
+    np.testing.assert_array_equal(shift["y_d"], ref["y_d"] + b.astype(np.float64))
+    assert np.abs(oracle.output_affine(ref, b, a)["y_d"] - want).max() > 1e-3
+
+
 def test_channel_major_wrapper_is_the_per_token_definition():
     """quantize_act_nchw must treat x[b, :, h, w] as one token (Supp. S1.1's 4-D branch), with token
     index (b*H + h)*W + w: checked token by token with plain indexing, no transpose."""
