@@ -46,7 +46,7 @@ typedef enum {
     TDQ_ERR_DEVICE_TIMEOUT = 6  /* a bounded device-side wait ran out (see workspace status) */
 } tdq_status;
 
-typedef enum { TDQ_F32 = 0, TDQ_BF16 = 1 } tdq_dtype;
+typedef enum { TDQ_F32 = 0, TDQ_BF16 = 1, TDQ_F16 = 2 /* outputs of the linear layer only */ } tdq_dtype;
 
 /* Which DCRP bounds take part in the projection (Algorithm S1 step 4; the ablation
  * variants of Table S6).  Both = COD-TDQ, neither = DSTG only. */
@@ -160,7 +160,8 @@ tdq_status tdq_fold_output_affine(const float* wscale, const float* bias, const 
  *   xcodes [M, I_pad/2], xscale [M, K], wcodes [O, I_pad/2], wscale [O], bias NULL or [O].
  *   I_pad must be a multiple of group_size; group_size a multiple of 32 (the integer
  *   tensor-core instruction contracts 32 codes at a time), at most 4096.
- *   y      [M, O], y_dtype (float32 or bf16), rows y_row_stride elements apart (>= O).
+ *   y      [M, O], y_dtype (float32, bf16 or fp16; the 16-bit types are rounded to nearest even from the
+ *          float32 result), rows y_row_stride elements apart (>= O).
  *   acc_debug  NULL, or [M, O, K] int32 receiving every group's integer dot product
  *              (for tests; slows the kernel down).
  *   workspace  at least tdq_linear_workspace_bytes() bytes, 16-byte aligned.  Holds the

@@ -17,7 +17,7 @@ if not os.path.exists(LIB_PATH):
 _lib = ctypes.CDLL(LIB_PATH)
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_DEVICE_TIMEOUT = range(7)
-F32, BF16 = 0, 1
+F32, BF16, F16 = 0, 1, 2
 ENABLE_C1, ENABLE_C2, POW2_STEP = 1, 2, 4
 
 # every symbol include/tdq.h declares
@@ -113,7 +113,9 @@ def _dtype_id(t: torch.Tensor) -> int:
         return F32
     if t.dtype == torch.bfloat16:
         return BF16
-    raise TypeError("tdq takes float32 or bfloat16 tensors, got %s" % t.dtype)
+    if t.dtype == torch.float16:
+        return F16          # outputs of the linear layer only; the library refuses it elsewhere
+    raise TypeError("tdq takes float32, bfloat16 or (for outputs) float16 tensors, got %s" % t.dtype)
 
 
 def _stream(t: torch.Tensor):

@@ -64,7 +64,7 @@ extern "C" tdq_status tdq_quant_linear_host(const void* x_host, tdq_dtype x_dtyp
     if (!x_host || !y_host || !x_dev || !codes_dev || !scale_dev || !y_dev || !p) return TDQ_ERR_INVALID_ARG;
     if (B < 0 || N < 0 || C <= 0 || O <= 0) return TDQ_ERR_INVALID_ARG;
     if (x_dtype != TDQ_F32 && x_dtype != TDQ_BF16) return TDQ_ERR_INVALID_ARG;
-    if (y_dtype != TDQ_F32 && y_dtype != TDQ_BF16) return TDQ_ERR_INVALID_ARG;
+    if (y_dtype != TDQ_F32 && y_dtype != TDQ_BF16 && y_dtype != TDQ_F16) return TDQ_ERR_INVALID_ARG;
     // every check of the two calls that does not depend on a chunk's pointers is made here, before anything is
     // queued: a refusal must leave the streams untouched
     tdq_status chk = check_act_args(x_dev, x_dtype, B, N, C, C, p);
@@ -86,7 +86,7 @@ extern "C" tdq_status tdq_quant_linear_host(const void* x_host, tdq_dtype x_dtyp
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
     HostPipe* hp = host_pipe();
     if (!hp) return TDQ_ERR_CUDA;
-    const int64_t xe = x_dtype == TDQ_BF16 ? 2 : 4, ye = y_dtype == TDQ_BF16 ? 2 : 4;
+    const int64_t xe = x_dtype == TDQ_BF16 ? 2 : 4, ye = y_dtype == TDQ_F32 ? 4 : 2;
     const int64_t g = p->group_size;
     const int64_t K = (C + g - 1) / g, I_pad = K * g;
     int64_t rows_per = (M + kHostChunks - 1) / kHostChunks;

@@ -680,10 +680,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                 o2 = __fmaf_rn(s4.z, o2, b4.z);
                 o3 = __fmaf_rn(s4.w, o3, b4.w);
                 if (YBF16) {       // columns 4 j .. 4 j + 3: half of chunk j / 2
-                    __nv_bfloat162 lo = __floats2bfloat162_rn(o0, o1);
-                    __nv_bfloat162 hi = __floats2bfloat162_rn(o2, o3);
                     *reinterpret_cast<uint2*>(strip + ((((uint32_t)j >> 1) ^ swz) << 4) + ((uint32_t)j & 1u) * 8) =
-                        make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+                        make_uint2(pack16(o0, o1, a.y_f16), pack16(o2, o3, a.y_f16));
                 } else {
                     *reinterpret_cast<float4*>(strip + (((uint32_t)j ^ swz) << 4)) = make_float4(o0, o1, o2, o3);
                 }
@@ -879,7 +877,9 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
     if (fx && (!fx->x || group_size != 32 || acc_debug)) return TDQ_ERR_UNSUPPORTED;
     if (!wcodes || !wscale || !y) return TDQ_ERR_INVALID_ARG;
     if (M < 0 || O <= 0 || I_pad <= 0 || y_row_stride < O) return TDQ_ERR_INVALID_ARG;
-    if (y_dtype != TDQ_F32 && y_dtype != TDQ_BF16) return TDQ_ERR_INVALID_ARG;
+    if (y_dtype != TDQ_F32 && y_dtype != TDQ_BF16 && y_dtype != TDQ_F16) return TDQ_ERR_INVALID_ARG;
+    const bool y_f16 = y_dtype == TDQ_F16;
+    if (y_f16) y_dtype = TDQ_BF16;      // the 16-bit kernels serve both types; a flag picks the conversion
     if (group_size <= 0 || I_pad % group_size) return TDQ_ERR_INVALID_ARG;
     if (group_size % 32 || group_size > 4096) return TDQ_ERR_UNSUPPORTED;
     if (I_pad / 2 > INT32_MAX) return TDQ_ERR_INVALID_ARG;
@@ -955,13 +955,14 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
     // g = 32 with y that tensor stores can write goes to the kernel built for it (tdq_linear_g32.cu)
     const bool use_g32 = !i8 && !pow2_steps && !fx && y_tma;
     if (y_tma && encode_y_map(&ymap, y, y_dtype == TDQ_BF16, M, O, y_row_stride, half_strips ? kCols / 2 : kCols,
-                              use_g32 ? kBM : 32))
+                              use_g32 ? kBM : 32, y_f16))
         a.tma_ok = 1;
     else if (narrow_strips)
         return TDQ_ERR_CUDA;   // the plan counted on the tensor store
     a.staging_bytes = (uint32_t)staging_bytes;
     a.half_strips = half_strips ? 1 : 0;
     a.out_scale = i8 ? 0.00390625f : 262144.0f;
+    a.y_f16 = y_f16 ? 1 : 0;
     a.xcodes = xcodes; a.xscale = xscale; a.row_bytes = e.row_bytes; a.unpack_a = unpack_a ? 1 : 0;
     a.pair_groups = (i8 && a.steps_per_grp % kChunk == 0 && a.Kg >= 2) ? 1 : 0;
     a.x = fx ? fx->x : nullptr;

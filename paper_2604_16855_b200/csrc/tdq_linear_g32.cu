@@ -373,13 +373,11 @@ __global__ void __launch_bounds__(kThreadsG32, 1) w4a4_g32_kernel(const LinArgs 
                             unpack2(yacc[16 * hh + ((4 * j + 2) ^ kAccSwap)], o[4], o[5]);
                             unpack2(yacc[16 * hh + ((4 * j + 3) ^ kAccSwap)], o[6], o[7]);
                             const float4 sa = s4[2 * j], sb = s4[2 * j + 1], ba = b4[2 * j], bb = b4[2 * j + 1];
-                            __nv_bfloat162 h0 = __floats2bfloat162_rn(__fmaf_rn(sa.x, o[0], ba.x), __fmaf_rn(sa.y, o[1], ba.y));
-                            __nv_bfloat162 h1 = __floats2bfloat162_rn(__fmaf_rn(sa.z, o[2], ba.z), __fmaf_rn(sa.w, o[3], ba.w));
-                            __nv_bfloat162 h2 = __floats2bfloat162_rn(__fmaf_rn(sb.x, o[4], bb.x), __fmaf_rn(sb.y, o[5], bb.y));
-                            __nv_bfloat162 h3 = __floats2bfloat162_rn(__fmaf_rn(sb.z, o[6], bb.z), __fmaf_rn(sb.w, o[7], bb.w));
-                            sts128(row_s + (((uint32_t)j ^ (((uint32_t)lane >> 1) & 3u)) << 4), *reinterpret_cast<uint32_t*>(&h0),
-                                   *reinterpret_cast<uint32_t*>(&h1), *reinterpret_cast<uint32_t*>(&h2),
-                                   *reinterpret_cast<uint32_t*>(&h3));
+                            sts128(row_s + (((uint32_t)j ^ (((uint32_t)lane >> 1) & 3u)) << 4),
+                                   pack16(__fmaf_rn(sa.x, o[0], ba.x), __fmaf_rn(sa.y, o[1], ba.y), a.y_f16),
+                                   pack16(__fmaf_rn(sa.z, o[2], ba.z), __fmaf_rn(sa.w, o[3], ba.w), a.y_f16),
+                                   pack16(__fmaf_rn(sb.x, o[4], bb.x), __fmaf_rn(sb.y, o[5], bb.y), a.y_f16),
+                                   pack16(__fmaf_rn(sb.z, o[6], bb.z), __fmaf_rn(sb.w, o[7], bb.w), a.y_f16));
                         }
                     }
                 }

@@ -4,6 +4,7 @@
 // power-of-two variants) and tdq_linear_g32.cu (the g = 32 kernel).
 #pragma once
 #include <cuda.h>
+#include <cuda_fp16.h>
 #include <cstring>
 #include <type_traits>
 
@@ -65,6 +66,7 @@ struct LinArgs {
     uint32_t* status;
     int32_t tma_ok;            // y can be written with bulk tensor stores (16-byte aligned base and row pitch)
     float out_scale;           // 2^18 (E4M3 route) or 2^-8 (int8 route)
+    int32_t y_f16;             // 16-bit output is fp16 (else bf16); the kernels' 16-bit instances serve both
     // resident A without the fused producer: the promotion warps unpack the item's codes themselves
     const uint8_t* xcodes;
     const float* xscale;
@@ -310,6 +312,16 @@ __device__ __forceinline__ void fma2(uint64_t& acc, uint64_t v, uint64_t d) {
     asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(v), "l"(d));
 }
 
+// two floats -> one word of two bf16 or two fp16 (round to nearest even), low half first
+__device__ __forceinline__ uint32_t pack16(float lo, float hi, int f16) {
+    if (f16) {
+        __half2 h = __floats2half2_rn(lo, hi);
+        return *reinterpret_cast<uint32_t*>(&h);
+    }
+    __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&b);
+}
+
 // shared memory by 32-bit shared-window address
 __device__ __forceinline__ uint32_t lds32(uint32_t addr) {
     uint32_t v;
@@ -385,7 +397,7 @@ typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint3
                                       const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                       CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 bool encode_y_map(CUtensorMap* map, void* y, bool bf16, int64_t M, int64_t O, int64_t y_row_stride, int box_cols,
-                  int box_rows = 32) {
+                  int box_rows = 32, bool f16 = false) {
     static const TensorMapEncodeFn encode = [] {
         void* fn = nullptr;
         cudaDriverEntryPointQueryResult res;
@@ -401,7 +413,7 @@ bool encode_y_map(CUtensorMap* map, void* y, bool bf16, int64_t M, int64_t O, in
     const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
     const bool rows64 = (size_t)box_cols * esz == 64;   // 64-byte strip rows (else 128)
     const cuuint32_t elem_strides[2] = {1u, 1u};
-    return encode(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, y, dims, strides, box,
+    return encode(map, bf16 ? (f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16) : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, y, dims, strides, box,
                   elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, rows64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
                   CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }

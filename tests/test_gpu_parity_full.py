@@ -265,3 +265,34 @@ def test_affine_output_correction_folded_into_the_constants(tdq, with_bias, with
                                bias=np.zeros(O, np.float32) if bias is None else bias)
     # three more roundings than the plain layer (a_o s_o, a_o bias_o, + b_o), counted against the size of the terms
     compare_y(y.cpu().numpy(), ref, case.C // 32 + 3)
+
+
+# ---------------------------------------------------------------------------------------
+# fp16 output (rounded to nearest even from the float32 result), on both linear kernels and the fused call
+
+@pytest.mark.parametrize("idx,rows,g,fused", [(3, 1500, 32, False), (3, 700, 64, False), (2, 3000, 32, True), (1, 256, 32, False)])
+def test_fp16_output(tdq, idx, rows, g, fused):
+    case = si.config(idx)
+    x = case.x.reshape(-1, case.C)[:rows]
+    bias = np.linspace(-0.3, 0.3, case.O).astype(np.float32)
+    xt = to_cuda(x, bf16=case.x_is_bf16)
+    wc, ws = tdq.quantize_weight(to_cuda(case.w), pad_to=g)
+    p = tdq.act_params(g=g)
+    if fused:
+        y = tdq.quant_linear_fused(xt, wc, ws, to_cuda(bias), p, out_dtype=torch.float16)
+    else:
+        codes, scale = tdq.quantize_act(xt, p)
+        y = tdq.w4a4_linear(codes, scale, wc, ws, to_cuda(bias), g=g, out_dtype=torch.float16)
+        y32 = tdq.w4a4_linear(codes, scale, wc, ws, to_cuda(bias), g=g)
+        assert torch.equal(y, y32.to(torch.float16))          # exactly the float32 result rounded once
+    assert y.dtype == torch.float16
+    xa, wq = oracle.quantize_act(x, g=g), oracle.quantize_weight(case.w, pad_to=g)
+    ref = oracle.w4a4_linear(xa["codes"], xa["scale"], wq["codes"], wq["scale"], bias=bias, g=g)
+    # one fp16 rounding on top of the float32 rule: 2^-11 relative, or half the spacing of fp16 subnormals (2^-24)
+    # for the outputs of the low-amplitude tokens, which fall below fp16's smallest normal number
+    yn = y.float().cpu().numpy().astype(np.float64)
+    small = np.abs(ref["y_d"]) < 2.0 ** -14
+    ref_n = dict(y_d=np.where(small, yn, ref["y_d"]), t_abs=ref["t_abs"])
+    compare_y(yn, ref_n, case.C // g + 1, out_eps=2.0 ** -11)
+    tol_small = np.maximum(1e-5 * np.abs(ref["y_d"]), (case.C // g + 3) * 2.0 ** -24 * ref["t_abs"]) + 2.0 ** -25
+    assert (np.abs(yn - ref["y_d"])[small] <= tol_small[small]).all()
