@@ -41,9 +41,43 @@ METRIC = "quantizer GB/s and W4A4 linear TOPS at 1 B200, % of HBM / INT8 rooflin
 L2_BYTES = 126 * 2 ** 20
 
 
-# DRAM bytes (read + write) of one w4a4_gemm_kernel launch on cfg4 from the ncu capture summarised in
-# profiles/w4a4_gemm_kernel_cfg4.md; reported only for that workload and output type.
-GEMM_DRAM_TRAFFIC_CFG4 = 179.0e6
+def kernel_source_hash(files):
+    """sha256 over the named source files of the package's csrc directory, in the given order."""
+    import hashlib
+    h = hashlib.sha256()
+    for name in files:
+        with open(os.path.join(ROOT, "paper_2604_16855_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def profiled_traffic(kernel, workload_name, files):
+    """DRAM bytes per launch of `kernel` on `workload_name` from the committed profile summary, or None.  A summary
+    counts only while the kernel's sources still hash to what the summary records (the counters were taken on that
+    code); its lines `kernel:`, `workload:`, `dram_bytes_per_launch:` and `kernel_source_sha256:` are read."""
+    d = os.path.join(ROOT, "profiles")
+    if not os.path.isdir(d):
+        return None
+    want = kernel_source_hash(files)
+    for name in sorted(os.listdir(d)):
+        fields = {}
+        try:
+            for line in open(os.path.join(d, name)):
+                if ":" in line:
+                    k, v = line.split(":", 1)
+                    fields[k.strip().strip("`*- ")] = v.strip().strip("`* ")
+        except OSError:
+            continue
+        if fields.get("kernel") == kernel and fields.get("workload") == workload_name and \
+                fields.get("kernel_source_sha256") == want:
+            try:
+                return float(fields["dram_bytes_per_launch"])
+            except (KeyError, ValueError):
+                return None
+    return None
+
+
+LINEAR_G32_SOURCES = ["tdq_linear_g32.cu", "tdq_tc.cuh", "tdq_linear.cu"]
 
 
 def load_peaks():
@@ -139,6 +173,18 @@ def cpu_oracle_leg(case, rows, repeats=1):
                 quant_gbs=quant_bytes(x.shape[0], case.C, esize) / best_q / 1e9,
                 linear_tops=2.0 * x.shape[0] * case.C * case.O / best_l / 1e12,
                 cores=oracle.num_threads())
+
+
+def cpu_oracle_single_thread(workload_name, rows):
+    """The same oracle leg on one host thread (a child process, because the thread count of the oracle's OpenMP
+    runtime is fixed when it starts)."""
+    env = dict(os.environ, OMP_NUM_THREADS="1")
+    try:
+        r = subprocess.run([sys.executable, os.path.abspath(__file__), "--oracle-leg", str(rows), "--workload", workload_name],
+                           env=env, capture_output=True, text=True, timeout=600)
+        return json.loads(r.stdout.strip().splitlines()[-1])
+    except (subprocess.SubprocessError, ValueError, IndexError, OSError):
+        return None
 
 
 def run_reference(args):
@@ -458,6 +504,34 @@ def run_tdq(args):
         q_ms = sum(e[0].elapsed_time(e[1]) for e in evs) * args.steps / n_ev
         l_ms = sum(e[1].elapsed_time(e[2]) for e in evs) * args.steps / n_ev
 
+    # Sustained leg: the same step graph replayed for about two seconds with the clock sampler running.  The
+    # 20-step region above lasts a few milliseconds, too short for a 100 ms sampler and for the power cap to act;
+    # here the step time is read beside the SM clock it ran at, and their product (SM clocks per step) is what
+    # stays comparable when the clock moves.
+    sustained = None
+    if G and rank == 0 and world == 1:
+        n_rep = max(1, int(2.0 / max(1e-6, (total_ms / args.steps) * 1e-3 * G)))
+        s2 = ClockSampler(local)
+        s2.start()
+        time.sleep(0.25)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n_rep):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        c2 = s2.stop()
+        ms_step = e0.elapsed_time(e1) / (n_rep * G)
+        sustained = dict(seconds=e0.elapsed_time(e1) * 1e-3, steps=n_rep * G, ms_per_step=ms_step, clocks=c2,
+                         sm_clocks_per_step=(ms_step * 1e-3 * c2["sm_mhz"] * 1e6) if c2.get("sm_mhz") else None)
+    # warm-cache figures: the same call on one buffer set, launched back to back (inputs stay in L2 where they fit)
+    warm = None
+    if G and world == 1:
+        warm = dict(
+            quantize_ms=time_graph(lambda i: tdq.quantize_act(xs[0], params, codes=codes[0], scale=scales[0]), 16),
+            linear_ms=time_graph(lambda i: tdq.w4a4_linear(codes[0], scales[0], wcodes, wscale, y=ys[0], workspace=wsp), 8))
+
     # end to end: pinned host X in, host Y out, through the host-buffer entry point
     xh = x_host.pin_memory()
     yh = torch.empty((M, O), dtype=torch.float32).pin_memory()
@@ -558,6 +632,16 @@ def run_tdq(args):
         l_gbs = lb * K / (l_ms * 1e-3) / 1e9
         l_tops = ops * K / (l_ms * 1e-3) / 1e12
         int8_peak = 2.0 * peaks["bf16_tflops"]            # nominal int8 : bf16 ratio on the measured bf16 peak
+        # the library's own figure: clocks per 128 x 128 x 32 instruction with operands resident in shared memory
+        mma_peak = None
+        if world == 1:
+            n_sm = torch.cuda.get_device_properties(dev).multi_processor_count
+            clk_max = (clocks or {}).get("sm_max_mhz") or 1965.0
+            mma_peak = {}
+            for label, kind in (("e4m3_f32acc", False), ("int8_int32acc", True)):
+                cpm = tdq.measure_mma_clocks(kind, 8192, dev)
+                mma_peak[label] = dict(clocks_per_mma=cpm, tops_at_max_clock=2.0 * 128 * 128 * 32 * n_sm * clk_max * 1e6 / cpm / 1e12)
+            mma_peak["sm_max_mhz"] = clk_max
         q_kernel = dict(name="tdq_quantize_act", ms=q_ms / K, gbs=q_gbs, frac_hbm=q_gbs / peaks["hbm_gbs"],
                         frac_hbm_8tbs=q_gbs / 8000.0, algorithmic_bytes=qb)
         timing = ("events around launches of this call alone, replayed from a CUDA graph over rotating buffers" if G
@@ -570,13 +654,17 @@ def run_tdq(args):
                         algorithmic_bytes=lb, ops=ops,
                         bound="hbm" if lb / peaks["hbm_gbs"] / 1e9 > ops / int8_peak / 1e12 else "tensor")
         l_kernel["timing"] = timing
+        if mma_peak:
+            l_kernel["frac_int8_measured_issue_rate"] = l_tops / mma_peak["e4m3_f32acc"]["tops_at_max_clock"]
+        if warm:
+            q_kernel["ms_warm"], l_kernel["ms_warm"] = warm["quantize_ms"], warm["linear_ms"]
         if l_iso_ms:
             l_kernel.update(ms_between_event_nodes_in_step=l_iso_ms)
         if l_ms >= q_ms:
             if l_kernel["bound"] == "hbm":
                 roof = dict(kernel="tdq_w4a4_linear", bound="hbm", achieved=l_gbs, peak=peaks["hbm_gbs"],
                             unit="GB/s", frac=l_gbs / peaks["hbm_gbs"],
-                            traffic=GEMM_DRAM_TRAFFIC_CFG4 if case.name.startswith("cfg4") else None)
+                            traffic=profiled_traffic("w4a4_g32_kernel", args.workload, LINEAR_G32_SOURCES))
             else:
                 roof = dict(kernel="tdq_w4a4_linear", bound="tensor", achieved=l_tops, peak=int8_peak,
                             unit="TOP/s", frac=l_tops / int8_peak, traffic=None)
@@ -596,7 +684,7 @@ def run_tdq(args):
                                parallelism="rows sharded, %d replica(s)" % world),
                    kernels=dict(quantize_act=q_kernel, quantize_act_nchw=q_nchw, w4a4_linear=l_kernel, w4a4_linear_pow2=pow2, fused=fused, sweep_cfg5=sweep, configs_1_to_3=small, compute_probe=probe,
                                 step_tokens_per_s=world * M * K / (total_ms * 1e-3)),
-                   roofline=roof, clocks=clocks, gpu_launches=int(launches),
+                   roofline=roof, clocks=clocks, sustained=sustained, mma_peak=mma_peak, gpu_launches=int(launches),
                    e2e=dict(value=e2e_value, unit="GB/s", ms_per_step=e2e_ms / e2e_steps,
                             h2d_bytes_per_step=int(M * C * esize), d2h_bytes_per_step=int(M * O * 4),
                             api="tdq_quant_linear_host"))
@@ -607,6 +695,10 @@ def run_tdq(args):
                                               % (leg["rows"], M, case.name),
                                        linear_tops=leg["linear_tops"], quant_s=leg["quant_s"],
                                        linear_s=leg["linear_s"])
+            one = cpu_oracle_single_thread(args.workload, min(M, 1024))
+            if one:
+                out["cpu_baseline"]["single_thread"] = dict(value=one["quant_gbs"], unit="GB/s", linear_tops=one["linear_tops"],
+                                                            sample="first %d token rows" % one["rows"])
         print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
@@ -622,8 +714,12 @@ def main():
     ap.add_argument("--cpu-rows", type=int, default=18464)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the fused-call and 32-layer sweep legs")
+    ap.add_argument("--oracle-leg", type=int, default=0, help=argparse.SUPPRESS)
     ap.add_argument("--eager", action="store_true", help="launch every timed step from the host instead of replaying a CUDA graph")
     args = ap.parse_args()
+    if args.oracle_leg:                    # child of cpu_oracle_single_thread
+        print(json.dumps(cpu_oracle_leg(workload(args.workload), args.oracle_leg)))
+        return
     if args.steps is None:
         args.steps = 10 if args.impl == "reference" else 1000
     if args.impl == "reference":

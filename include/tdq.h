@@ -299,6 +299,20 @@ tdq_status tdq_quantize_status(void* cuda_stream, uint32_t* detail /* HOST */);
  */
 tdq_status tdq_selftest_wait_timeout(int32_t which, int64_t limit_cycles, void* workspace, void* cuda_stream);
 
+/*
+ * Measures how fast the tensor cores of the current device run the instruction the linear layer is built on (no
+ * counterpart in the paper; the benchmark uses it for its own dense 8-bit peak): one thread block per SM issues
+ * n_mma tcgen05.mma instructions of shape 128 x 128 x 32 on operands resident in shared memory, with nothing else
+ * running, and the slowest SM's clocks per instruction come back in *clocks_per_mma (HOST).  Peak operations per
+ * second = 2 * 128 * 128 * 32 * SMs * SM clock / clocks_per_mma.
+ *   integer_kind  0: E4M3 operands, float32 accumulator (the g = 32 route); 1: int8 operands, int32 accumulator.
+ *   n_mma         a multiple of 4 between 4 and 2^22.
+ *   scratch       device memory, 16-byte aligned, at least 16 bytes per SM.
+ * The call waits for its kernel (it is a measurement, not part of the path).
+ */
+tdq_status tdq_measure_mma_clocks(int32_t integer_kind, int32_t n_mma, void* scratch, size_t scratch_bytes,
+                                  double* clocks_per_mma /* HOST */, void* cuda_stream);
+
 /* Static description of a status code. */
 const char* tdq_status_string(tdq_status s);
 

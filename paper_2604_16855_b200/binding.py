@@ -24,7 +24,7 @@ ENABLE_C1, ENABLE_C2, POW2_STEP = 1, 2, 4
 EXPORTS = ["tdq_default_act_params", "tdq_quantize_act", "tdq_quantize_weight", "tdq_w4a4_linear",
            "tdq_quant_linear_fused", "tdq_quant_linear_host", "tdq_quantize_act_nchw", "tdq_quantize_act_fixed", "tdq_w4a4_linear_pow2", "tdq_linear_workspace_bytes",
            "tdq_workspace_status", "tdq_status_string", "tdq_kernel_launch_count", "tdq_w4a4_linear_static",
-           "tdq_quantize_status", "tdq_selftest_wait_timeout", "tdq_fold_output_affine"]
+           "tdq_quantize_status", "tdq_selftest_wait_timeout", "tdq_fold_output_affine", "tdq_measure_mma_clocks"]
 
 
 class ActParams(ctypes.Structure):
@@ -68,6 +68,8 @@ _lib.tdq_selftest_wait_timeout.argtypes = [_i32, _i64, _vp, _vp]
 _lib.tdq_selftest_wait_timeout.restype = ctypes.c_int
 _lib.tdq_fold_output_affine.argtypes = [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _vp]
 _lib.tdq_fold_output_affine.restype = ctypes.c_int
+_lib.tdq_measure_mma_clocks.argtypes = [_i32, _i32, _vp, _sz, ctypes.POINTER(ctypes.c_double), _vp]
+_lib.tdq_measure_mma_clocks.restype = ctypes.c_int
 _lib.tdq_status_string.argtypes = [ctypes.c_int]
 _lib.tdq_status_string.restype = ctypes.c_char_p
 _lib.tdq_kernel_launch_count.argtypes = []
@@ -380,3 +382,14 @@ def fold_output_affine(wscale, bias, out_mul, out_add=None):
         _check(_lib.tdq_fold_output_affine(_ptr(wscale), _ptr(bias), _ptr(out_mul), _ptr(out_add), O, _ptr(ws2), _ptr(b2),
                                            _stream(wscale)), "tdq_fold_output_affine")
     return ws2, b2
+
+
+def measure_mma_clocks(integer_kind: bool, n_mma: int = 8192, device="cuda") -> float:
+    """tdq_measure_mma_clocks: clocks per 128 x 128 x 32 tensor-core instruction on the slowest SM of the device."""
+    dev = torch.device(device)
+    scratch = torch.zeros((16 * 1024,), dtype=torch.uint8, device=dev)
+    out = ctypes.c_double(0.0)
+    with torch.cuda.device(dev):
+        _check(_lib.tdq_measure_mma_clocks(1 if integer_kind else 0, n_mma, _ptr(scratch), scratch.numel(), ctypes.byref(out),
+                                           ctypes.c_void_p(torch.cuda.current_stream(dev).cuda_stream)), "tdq_measure_mma_clocks")
+    return float(out.value)

@@ -16,7 +16,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libtdq.so")
-SOURCES = ["tdq_quantize_act.cu", "tdq_quantize_weight.cu", "tdq_linear.cu", "tdq_linear_g32.cu", "tdq_fused.cu", "tdq_api.cu"]
+SOURCES = ["tdq_quantize_act.cu", "tdq_quantize_weight.cu", "tdq_linear.cu", "tdq_linear_g32.cu", "tdq_fused.cu", "tdq_api.cu", "tdq_peak.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "--ftz=false", "--prec-div=true", "--prec-sqrt=true"]

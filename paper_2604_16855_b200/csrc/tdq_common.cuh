@@ -6,6 +6,7 @@
 #include <stdint.h>
 
 #include <atomic>
+#include <utility>
 #include <cmath>
 
 #include "../../include/tdq.h"
@@ -68,6 +69,31 @@ inline int current_device_sm_count(int* device = nullptr) {
 // true once `done` has the device's bit; the caller sets the attribute when this returns false and then calls mark
 inline bool device_marked(const std::atomic<uint64_t>& done, int dev) { return (done.load(std::memory_order_acquire) >> dev) & 1u; }
 inline void mark_device(std::atomic<uint64_t>& done, int dev) { done.fetch_or(1ull << dev, std::memory_order_release); }
+
+// Programmatic dependent launch.  The hot-path kernels are launched with the attribute that lets a grid start
+// while its predecessor in the stream is still draining; each of them executes pdl_wait() in every thread before its
+// first access to global memory (the wait returns when the preceding grids have completed and their writes are
+// visible), so only block scheduling, shared-memory set-up and barrier initialisation overlap the predecessor's
+// tail.  pdl_trigger() tells the scheduler that the next grid may be brought in.  Inside a captured graph the
+// same launches become programmatic edges.  Kernels launched the ordinary way need neither call.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+#endif
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 
 inline tdq_status cuda_status(cudaError_t e) { return e == cudaSuccess ? TDQ_OK : TDQ_ERR_CUDA; }
 

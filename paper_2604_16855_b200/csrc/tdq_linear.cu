@@ -83,6 +83,8 @@ struct ExpandArgs {
 // One CTA rewrites one (128-row block, 4 K-steps) piece: thread t takes row t / 4 and K-step t % 4.
 template <bool I8>
 __global__ void __launch_bounds__(kExpandThreads) expand_kernel(ExpandArgs a) {
+    pdl_wait();
+    pdl_trigger();
     const int piece = blockIdx.x;
     if (piece == 0 && threadIdx.x < 4) a.status[threadIdx.x] = 0u;   // saves a separate memset in front of every call
     const int blk = piece / a.n_chunks, kc = piece % a.n_chunks;
@@ -232,6 +234,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    pdl_wait();          // barrier set-up and the TMEM allocation overlap the tail of the kernel before this one
+    pdl_trigger();
     const uint32_t tmem_base = c->tmem_base;
 
     const int n_items = a.tiles_m * a.n_parts;
@@ -988,18 +992,16 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
         if (cudaMemsetAsync(workspace, 0, 16, stream) != cudaSuccess) return TDQ_ERR_CUDA;
         expand_pow2_kernel<<<pieces, kExpandThreads, 0, stream>>>(e, act_group / 32, (int32_t)(I_pad / act_group));
     }
-    else if (i8)
-        expand_kernel<true><<<pieces, kExpandThreads, 0, stream>>>(e);
-    else
-        expand_kernel<false><<<pieces, kExpandThreads, 0, stream>>>(e);
+    else if ((i8 ? launch_pdl(expand_kernel<true>, dim3(pieces), dim3(kExpandThreads), 0, stream, e)
+                 : launch_pdl(expand_kernel<false>, dim3(pieces), dim3(kExpandThreads), 0, stream, e)) != cudaSuccess)
+        return TDQ_ERR_CUDA;
     if (cudaGetLastError() != cudaSuccess) return TDQ_ERR_CUDA;
     g_launch_count.fetch_add(1, std::memory_order_relaxed);
 
     const int64_t items = p.tiles_m * p.n_parts;
     const unsigned grid = (unsigned)(items < n_sm ? items : n_sm);
     if (use_g32 && a.tma_ok) return launch_linear_g32(a, ymap, p.smem_bytes, grid, ybf, dbg, stream);
-    kernel<<<grid, kThreads, p.smem_bytes, stream>>>(a, ymap);
-    if (cudaGetLastError() != cudaSuccess) return TDQ_ERR_CUDA;
+    if (launch_pdl(kernel, dim3(grid), dim3(kThreads), p.smem_bytes, stream, a, ymap) != cudaSuccess) return TDQ_ERR_CUDA;
     g_launch_count.fetch_add(1, std::memory_order_relaxed);
     return TDQ_OK;
 }

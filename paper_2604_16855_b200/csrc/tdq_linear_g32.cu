@@ -106,6 +106,8 @@ __global__ void __launch_bounds__(kThreadsG32, 1) w4a4_g32_kernel(const LinArgs 
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    pdl_wait();          // barrier set-up and the TMEM allocation overlap the tail of the kernel before this one
+    pdl_trigger();
     const uint32_t tmem_base = c->tmem_base;
 
     const int n_items = a.tiles_m * a.n_parts;
@@ -515,8 +517,7 @@ tdq_status launch_linear_g32(const LinArgs& a, const CUtensorMap& ymap, uint32_t
     if (ybf && dbg) kernel = w4a4_g32_kernel<true, true>;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit) != cudaSuccess)
         return TDQ_ERR_CUDA;
-    kernel<<<grid, kThreadsG32, smem_bytes, stream>>>(a, ymap);
-    if (cudaGetLastError() != cudaSuccess) return TDQ_ERR_CUDA;
+    if (launch_pdl(kernel, dim3(grid), dim3(kThreadsG32), smem_bytes, stream, a, ymap) != cudaSuccess) return TDQ_ERR_CUDA;
     g_launch_count.fetch_add(1, std::memory_order_relaxed);
     return TDQ_OK;
 }

@@ -152,6 +152,8 @@ __global__ void __launch_bounds__(kFastThreads) act_g32_kernel(ActArgs a) {
     constexpr int kSwzMask = kChunks - 1;
     __shared__ __align__(16) uint4 tile[kFastThreads * kChunks];
 
+    pdl_wait();
+    pdl_trigger();
     const int t = threadIdx.x;
     const int64_t g0 = (int64_t)blockIdx.x * kFastThreads;
     const char* xb = reinterpret_cast<const char*>(a.x);
@@ -266,6 +268,8 @@ __global__ void __launch_bounds__(kRingThreads) act_g32_ring_kernel(ActArgs a, i
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    pdl_wait();          // everything above overlaps the tail of the kernel before this one
+    pdl_trigger();
     const char* xb = reinterpret_cast<const char*>(a.x);
     if (t >= kFastThreads) {
         if (t == kFastThreads) {   // producer lane
@@ -325,8 +329,7 @@ cudaError_t launch_ring(const ActArgs& a, cudaStream_t st) {
     }
     const int64_t n_tiles = (a.total_groups + kFastThreads - 1) / kFastThreads;
     const int64_t grid = n_tiles < 2 * n_sm ? n_tiles : 2 * n_sm;
-    act_g32_ring_kernel<BF16, KZR, KB><<<(unsigned)grid, kRingThreads, smem, st>>>(a, n_tiles);
-    return cudaGetLastError();
+    return launch_pdl(act_g32_ring_kernel<BF16, KZR, KB>, dim3((unsigned)grid), dim3(kRingThreads), smem, st, a, n_tiles);
 }
 
 // every zero-bin rank of a group of 32 has its instance of the two row-major kernels
@@ -342,16 +345,14 @@ cudaError_t launch_fast(const ActArgs& a, cudaStream_t st) {
     if (a.k_base != 32 && (a.k_base < 29 || a.k_zr != 7)) {
         // any other pair of ranks: the instance that takes both at run time
         if (a.row_stride == a.C) return launch_ring<BF16, 0, 0>(a, st);
-        act_g32_kernel<BF16, 0, 0><<<grid, block, 0, st>>>(a);
-        return cudaGetLastError();
+        return launch_pdl(act_g32_kernel<BF16, 0, 0>, grid, block, 0, st, a);
     }
     if (a.k_base != 32) {        // percentile base radius: ranks 29..31 beside the default zero-bin rank
         switch (a.k_base) {
 #define TDQ_CASE(KB_)                                                                  \
             case KB_:                                                                  \
                 if (a.row_stride == a.C) return launch_ring<BF16, 7, KB_>(a, st);      \
-                act_g32_kernel<BF16, 7, KB_><<<grid, block, 0, st>>>(a);               \
-                return cudaGetLastError();
+                return launch_pdl(act_g32_kernel<BF16, 7, KB_>, grid, block, 0, st, a);
             TDQ_CASE(29) TDQ_CASE(30) TDQ_CASE(31)
 #undef TDQ_CASE
             default: return cudaErrorInvalidValue;
@@ -366,7 +367,7 @@ cudaError_t launch_fast(const ActArgs& a, cudaStream_t st) {
         }
     }
     switch (a.k_zr) {
-#define TDQ_CASE(KZ) case KZ: act_g32_kernel<BF16, KZ><<<grid, block, 0, st>>>(a); break;
+#define TDQ_CASE(KZ) case KZ: return launch_pdl(act_g32_kernel<BF16, KZ>, grid, block, 0, st, a);
         TDQ_ALL_RANKS
 #undef TDQ_CASE
         default: return cudaErrorInvalidValue;
