@@ -238,6 +238,15 @@ def whole_job_rate(units_per_rank, world, ms):
     return world * units_per_rank / (ms * 1e-3)
 
 
+def shard_rows(M, rank, world):
+    """The token rows [start, stop) rank `rank` of `world` takes when one batch is split over the ranks (rows are
+    independent, weights are replicated, nothing is exchanged): whole 128-row blocks, the remainder to the last ranks."""
+    blocks = (M + 127) // 128
+    lo = (blocks * rank) // world * 128
+    hi = M if rank == world - 1 else (blocks * (rank + 1)) // world * 128
+    return min(lo, M), min(hi, M)
+
+
 def graph_steps(K, nsets, cap=64):
     """Steps per graph: the largest divisor of K that is a multiple of the buffer rotation and at
     most `cap`; K itself (one graph, one replay) when there is none."""
@@ -509,7 +518,7 @@ def run_tdq(args):
     # here the step time is read beside the SM clock it ran at, and their product (SM clocks per step) is what
     # stays comparable when the clock moves.
     sustained = None
-    if G and rank == 0 and world == 1:
+    if G and rank == 0 and world == 1 and not args.no_extras:
         n_rep = max(1, int(2.0 / max(1e-6, (total_ms / args.steps) * 1e-3 * G)))
         s2 = ClockSampler(local)
         s2.start()
@@ -634,7 +643,7 @@ def run_tdq(args):
         int8_peak = 2.0 * peaks["bf16_tflops"]            # nominal int8 : bf16 ratio on the measured bf16 peak
         # the library's own figure: clocks per 128 x 128 x 32 instruction with operands resident in shared memory
         mma_peak = None
-        if world == 1:
+        if world == 1 and not args.no_extras:
             n_sm = torch.cuda.get_device_properties(dev).multi_processor_count
             clk_max = (clocks or {}).get("sm_max_mhz") or 1965.0
             mma_peak = {}
@@ -713,7 +722,7 @@ def main():
     ap.add_argument("--workload", default="cfg4", choices=["cfg1", "cfg2", "cfg3", "cfg4"])
     ap.add_argument("--cpu-rows", type=int, default=18464)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-extras", action="store_true", help="skip the fused-call and 32-layer sweep legs")
+    ap.add_argument("--no-extras", action="store_true", help="only the timed steps, the per-kernel timings and the end-to-end leg (for profiler runs)")
     ap.add_argument("--oracle-leg", type=int, default=0, help=argparse.SUPPRESS)
     ap.add_argument("--eager", action="store_true", help="launch every timed step from the host instead of replaying a CUDA graph")
     args = ap.parse_args()

@@ -49,6 +49,58 @@ def test_two_ranks_take_the_slowest_time_and_sum_the_work():
     assert abs(rate - 2 * 1000.0 / 11e-3) < 1e-6
 
 
+def _shard_worker(rank, world, port, out):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    sys.path.insert(0, ROOT)
+    import bench
+    import oracle
+    import synth_inputs as si
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    case = si.config3()
+    x = case.x.reshape(-1, case.C)[:1000]                # 1000 rows: the last rank gets a ragged block
+    wq = oracle.quantize_weight(case.w)                   # replicated on every rank
+    lo, hi = bench.shard_rows(x.shape[0], rank, world)
+    xa = oracle.quantize_act(x[lo:hi])
+    y = oracle.w4a4_linear(xa["codes"], xa["scale"], wq["codes"], wq["scale"])["y"]
+    parts = [None] * world
+    dist.all_gather_object(parts, (lo, hi, xa["codes"], xa["scale"], y))
+    if rank == 0:
+        parts.sort(key=lambda p: p[0])
+        assert parts[0][0] == 0 and parts[-1][1] == x.shape[0]
+        assert all(parts[i][1] == parts[i + 1][0] for i in range(world - 1)) and all(p[0] % 128 == 0 for p in parts)
+        full = oracle.quantize_act(x)
+        y_full = oracle.w4a4_linear(full["codes"], full["scale"], wq["codes"], wq["scale"])["y"]
+        ok = (np.array_equal(np.concatenate([p[2] for p in parts]), full["codes"])
+              and np.array_equal(np.concatenate([p[3] for p in parts]), full["scale"])
+              and np.array_equal(np.concatenate([p[4] for p in parts]), y_full))
+        out.put(ok)
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_ranks_shard_the_rows_and_reproduce_the_unsharded_result():
+    """Row shards through the whole path (here the oracle stands in for it, on CPU) concatenate to the unsharded
+    result bit for bit: the ranks exchange nothing but the finished outputs."""
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_shard_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    assert out.get(timeout=300) is True
+    for p in procs:
+        p.join(timeout=120)
+        assert p.exitcode == 0
+    import bench
+    for M, world in [(18464, 8), (256, 4), (100, 3), (1, 2)]:
+        spans = [bench.shard_rows(M, r, world) for r in range(world)]
+        assert spans[0][0] == 0 and spans[-1][1] == M and all(spans[i][1] == spans[i + 1][0] for i in range(world - 1))
+
+
 def test_graph_steps_divides_the_step_count_and_respects_the_buffer_rotation():
     import bench
     for K, nsets in [(1000, 2), (50, 2), (7, 2), (64, 3), (97, 2), (128, 4), (3, 2)]:
