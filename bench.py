@@ -77,7 +77,7 @@ def profiled_traffic(kernel, workload_name, files):
     return None
 
 
-LINEAR_G32_SOURCES = ["tdq_linear_g32.cu", "tdq_tc.cuh", "tdq_linear.cu"]
+LINEAR_G32_SOURCES = ["tdq_linear_g32.cu", "tdq_tc.cuh"]
 
 
 def load_peaks():
