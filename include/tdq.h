@@ -209,6 +209,8 @@ tdq_status tdq_w4a4_linear_pow2(const uint8_t* xcodes, const float* xscale, cons
  * aligned with a row pitch that is a multiple of 16 bytes, the zero-bin rank ceil(32 zr) == 7
  * when the C2 bound is enabled, and C <= 768 (a row block's operand bytes must fit in shared
  * memory).  Callers fall back to the two calls in those cases.
+ * Speed: on the benchmark workloads this call is not faster than the two calls it replaces (a tie on the
+ * smallest, about a third slower on the largest); its use is that activation codes never reach memory.
  */
 tdq_status tdq_quant_linear_fused(const void* x, tdq_dtype x_dtype, int64_t B, int64_t N, int64_t C,
                                   int64_t row_stride_elems, const tdq_act_params* p /* HOST */,
