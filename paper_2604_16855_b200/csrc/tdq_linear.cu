@@ -80,6 +80,16 @@ struct ExpandArgs {
     uint32_t* status;        // the workspace's status words, cleared here for the GEMM that follows
 };
 
+// Waits for this thread's outstanding TMEM loads; the 16 landing registers pass through as operands, so that no
+// use of them can be scheduled above the wait.
+__device__ __forceinline__ void tmem_ld_wait_on16(uint32_t* v) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]),
+                   "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15])
+                 :
+                 : "memory");
+}
+
 // One CTA rewrites one (128-row block, 4 K-steps) piece: thread t takes row t / 4 and K-step t % 4.
 template <bool I8>
 __global__ void __launch_bounds__(kExpandThreads) expand_kernel(ExpandArgs a) {
@@ -282,9 +292,11 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                     if (I8 && a.pair_groups) {   // (wide groups always take the integer instruction)
                         // two rings: this warp feeds the MMA warp of its parity through the stages of its parity, with
                         // the chunks of that warp's groups (group = steps_per_grp / 4 consecutive chunks of a tile)
-                        const int cpg = a.steps_per_grp / kChunk;
-                        for (int kc = 0; kc < n_chunks && ok; ++kc) {
-                            if (((kc / cpg) & 1) != warp) continue;
+                        // (pair_groups == 2: one group per tile, its chunks go to the two warps in turn)
+                        const int cpg = a.pair_groups == 2 ? 1 : a.steps_per_grp / kChunk;
+                        const int kc_step = a.pair_groups == 2 ? 2 : 1;
+                        for (int kc = a.pair_groups == 2 ? warp : 0; kc < n_chunks && ok; kc += kc_step) {
+                            if (a.pair_groups != 2 && ((kc / cpg) & 1) != warp) continue;
                             const uint32_t st = 2 * ps + (uint32_t)warp;
                             ok = mbar_wait_warp(&c->empty[st], pph ^ 1, c, a.status, 5u);
                             if (!ok) break;
@@ -336,6 +348,9 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
             const uint32_t tempty_s = smem_u32(&c->tempty[0]);
             const int n_steps = a.n_steps;
             // Group k of a tile uses TMEM slot k & 3, so a chunk of four steps always starts at slot 0.
+            // 5: one group per tile whose chunks the two warps take in turn, each into an accumulator of its own, which
+            // the promotion warps add (integer sums, so the split changes nothing): slots 0 and 1 for even tiles of this
+            // CTA, 2 and 3 for odd ones (SPLITQ);
             // mode 0: one instruction per group, two warps that take the even and the odd slots (DUAL); 3: two
             // instructions per group, two warps that take the first and the second group of a chunk (DUAL2);
             // 1: groups of a multiple of four steps, so that a chunk belongs to one group and is issued as
@@ -344,7 +359,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
             // other group width, one step at a time
             auto role = [&](auto mode_tag) {
                 constexpr int MODE = decltype(mode_tag)::value;
-                constexpr bool DUAL = MODE == 0, QUAD = MODE == 1, DUAL2 = MODE == 3, PAIRQ = MODE == 4;
+                constexpr bool DUAL = MODE == 0, QUAD = MODE == 1, DUAL2 = MODE == 3, PAIRQ = MODE == 4, SPLITQ = MODE == 5;
                 uint32_t s = 0, ph = 0, ib = 0, iu = 0;
                 bool ok = true;
                 // DUAL: this warp's two slots (me and me + 2), everything about them precomputed
@@ -355,7 +370,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                 uint32_t q_a = 1, q_b = 1;     // parity to wait for on tempty of each slot; a fresh barrier passes parity 1
                 // otherwise: one slot at a time
                 uint32_t qm = 0xFu;            // the same parities as a mask, bit = slot
-                uint32_t ps = 0, pph = 0;      // PAIRQ: position and phase in this warp's half of the ring (stages me, me + 2, ...)
+                uint32_t ps = 0, pph = 0;      // PAIRQ, SPLITQ: position and phase in this warp's half of the ring (stages me, me + 2, ...)
+                uint32_t tpar = 0;             // SPLITQ: parity of the tile among this CTA's tiles
                 const uint32_t n_mine = (n_stages + 1 - me) / 2;
                 for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
                     const int part = item % a.n_parts;
@@ -368,6 +384,37 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                         bool slot_ready = false;   // the early answer about the next slot, if it was yes
                         uint32_t a_lo = ares_lo;   // resident: walks through the item's A blocks
                         uint32_t grp = 0;          // PAIRQ: group of the tile this chunk belongs to
+                        if (SPLITQ) {
+                            // this warp's chunks only (me, me + 2, ...), with as little scalar work around the four
+                            // instructions as possible: a lone warp pays several clocks for every dependent instruction
+                            const int n_own = (n_chunks - (int)me + 1) / 2;
+                            const uint32_t gslot = 2u * tpar + me, d_tmem = tmem_base + gslot * kBN;
+                            const uint32_t full_s = smem_u32(&c->full[0]);
+                            uint32_t a_own = ares_lo + me * (uint32_t)(kChunk * (kBlock >> 4));
+                            for (int i = 0; i < n_own; ++i) {
+                                const uint32_t st = 2 * ps + me;
+                                if (!mbar_test_s(full_s + st * 8, pph)) {
+                                    ok = mbar_wait_warp(&c->full[st], pph, c, a.status, 4u);
+                                    if (!ok) break;
+                                }
+                                if (i == 0 && !mbar_test_s(tempty_s + gslot * 8, (qm >> gslot) & 1u)) {
+                                    ok = mbar_wait_warp(&c->tempty[gslot], (qm >> gslot) & 1u, c, a.status, 3u);
+                                    if (!ok) break;
+                                }
+                                tc_fence_after();
+                                const uint32_t b_st = ring_lo + st * stage_step;
+                                mma_issue4_if<I8>(lane0, d_tmem, resident ? a_own : b_st + a_in_stage, b_st, i == 0 ? 0u : 1u);
+                                if (i == n_own - 1) {
+                                    mma_commit_if(lane0, tfull_s + gslot * 8);
+                                    qm ^= 1u << gslot;
+                                }
+                                mma_commit_if(lane0, empty_s + st * 8);
+                                a_own += 2 * kChunk * (kBlock >> 4);
+                                if (++ps == n_mine) { ps = 0; pph ^= 1; }
+                            }
+                            tpar ^= 1u;
+                            continue;
+                        }
                         for (int k0 = 0; k0 < n_steps && ok; k0 += kChunk) {
                             if (PAIRQ) {
                                 // A group is spg / 4 consecutive chunks and belongs to the warp of its parity, which has
@@ -488,6 +535,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
             };
             if (spg == 1) role(std::integral_constant<int, 0>{});
             else if (spg == 2) role(std::integral_constant<int, 3>{});
+            else if (I8 && a.pair_groups == 2) role(std::integral_constant<int, 5>{});
             else if (I8 && a.pair_groups) role(std::integral_constant<int, 4>{});
             else if (spg % kChunk == 0) role(std::integral_constant<int, 1>{});
             else role(std::integral_constant<int, 2>{});
@@ -777,12 +825,66 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
             for (int q = 0; q < kLand / 2; ++q) fma2(yacc[(FUSED ? kLand / 2 : 0) + q], pack2(v[2 * q], v[2 * q + 1]), d2);
             return next_ready;
         };
+        // One group per tile in two accumulators (a.pair_groups == 2): slots UA and UA + 1 hold the sums over the even
+        // and the odd chunks of K.  Integer sums: their sum is the group's sum whatever the split.
+        auto consume_split = [&](auto u_tag) {
+            constexpr uint32_t UA = decltype(u_tag)::value, UB = UA + 1;
+            ok = mbar_wait_warp(&c->tfull[UA], p_full[UA], c, a.status, 2u);
+            if (ok) ok = mbar_wait_warp(&c->tfull[UB], p_full[UB], c, a.status, 2u);
+            p_full[UA] ^= 1u;
+            p_full[UB] ^= 1u;
+            if (!ok) return;
+            const uint32_t dbits = lds32(my_scale_s);
+            const uint64_t d2 = pack2(dbits, dbits);
+            tc_fence_after();
+            if (!FUSED) {
+                tmem_ld32(tmem_row_r + UA * kBN, v);
+                tmem_ld_wait();
+                uint32_t v2[kCols / 2];
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+#pragma unroll
+                    for (int q = 0; q < kCols / 2; ++q) v2[q] = 0u;
+                    tmem_ld16(tmem_row_r + UB * kBN + h * (kCols / 2), v2);
+                    tmem_ld_wait_on16(v2);
+#pragma unroll
+                    for (int q = 0; q < kCols / 2; ++q) v[h * (kCols / 2) + q] += v2[q];
+                }
+            }
+            tc_fence_before();                            // both slots are drained
+            __syncwarp();
+            mbar_arrive_lane0_s(tempty_s + UA * 8, lane);
+            mbar_arrive_lane0_s(tempty_s + UB * 8, lane);
+            if (DBG) {
+                const int64_t m = (int64_t)mt * kBM + row;
+                if (a.acc_debug && m < a.M) debug_store<I8>(a, v, m, n0, 0);
+            }
+            if (!FUSED) {
+#pragma unroll
+                for (int q = 0; q < kCols; ++q) v[q] = __float_as_uint((float)(int32_t)v[q]);
+#pragma unroll
+                for (int q = 0; q < kCols / 2; ++q) fma2(yacc[q], pack2(v[2 * q], v[2 * q + 1]), d2);
+            }
+        };
         const std::integral_constant<uint32_t, 0> u0{};
         const std::integral_constant<uint32_t, 1> u1{};
         const std::integral_constant<uint32_t, 2> u2{};
         const std::integral_constant<uint32_t, 3> u3{};
 
-        if (item < n_items) {
+        if (I8 && !FUSED && a.pair_groups == 2) {
+            if (item < n_items) {
+                begin_item();
+                if (ok) begin_tile();
+                uint32_t tpar = 0;
+#pragma unroll 1
+                while (ok && item < n_items) {
+                    if (tpar) consume_split(u2); else consume_split(u0);
+                    tpar ^= 1u;
+                    if (!ok) break;
+                    finish_tile();
+                }
+            }
+        } else if (item < n_items) {
             begin_item();
             if (ok) {
                 begin_tile();
@@ -969,6 +1071,8 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
     a.y_f16 = y_f16 ? 1 : 0;
     a.xcodes = xcodes; a.xscale = xscale; a.row_bytes = e.row_bytes; a.unpack_a = unpack_a ? 1 : 0;
     a.pair_groups = (i8 && a.steps_per_grp % kChunk == 0 && a.Kg >= 2) ? 1 : 0;
+    // one group per tile: the group's chunks go to the two MMA warps in turn, each with an accumulator of its own
+    if (i8 && !fx && a.Kg == 1 && a.steps_per_grp % kChunk == 0 && p.n_chunks >= 2) a.pair_groups = 2;
     a.x = fx ? fx->x : nullptr;
     a.x_stride = fx ? fx->row_stride : 0;
     a.seven_tau = fx ? fx->seven_tau : 0.0f;

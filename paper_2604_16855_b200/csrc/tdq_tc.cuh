@@ -72,7 +72,8 @@ struct LinArgs {
     const float* xscale;
     int32_t row_bytes;         // I_pad / 2
     int32_t unpack_a;
-    int32_t pair_groups;       // groups of a multiple of four steps, two or more per tile: the two MMA warps take them in turn
+    int32_t pair_groups;       // groups of a multiple of four steps: 1 = two or more per tile, the two MMA warps take them in turn;
+                               // 2 = one per tile, the warps take its chunks in turn into two accumulators
     // fused producer only: the activations themselves and the quantizer's parameters
     const void* x;
     int64_t x_stride;          // elements between rows of x

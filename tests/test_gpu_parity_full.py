@@ -296,3 +296,34 @@ def test_fp16_output(tdq, idx, rows, g, fused):
     compare_y(yn, ref_n, case.C // g + 1, out_eps=2.0 ** -11)
     tol_small = np.maximum(1e-5 * np.abs(ref["y_d"]), (case.C // g + 3) * 2.0 ** -24 * ref["t_abs"]) + 2.0 ** -25
     assert (np.abs(yn - ref["y_d"])[small] <= tol_small[small]).all()
+
+
+# ---------------------------------------------------------------------------------------
+# one group per token with a contraction of two or more ring stages: the two MMA-issuing warps take the
+# stages in turn, each into a TMEM accumulator of its own, and the promotion warps add the two integer sums.
+# Even and odd numbers of stages, several tiles per CTA (both pairs of accumulators), ragged edges.
+
+@pytest.mark.parametrize("M,C,O,bf16_out", [(300, 256, 200, False), (20000, 384, 384, False), (700, 640, 130, True),
+                                            (2100, 768, 1280, False), (129, 1024, 700, True), (5000, 128, 96, False)])
+def test_one_group_per_token_split_over_two_accumulators(tdq, M, C, O, bf16_out):
+    rng = np.random.RandomState(M + 3 * C + O)
+    x = (rng.normal(size=(M, C)) * np.exp(rng.normal(0, 1.0, size=(M, 1)))).astype(np.float32)
+    w = (rng.normal(size=(O, C)) * 0.05).astype(np.float32)
+    bias = rng.normal(size=(O,)).astype(np.float32) * 0.1
+    xa, wq = oracle.quantize_act(x, g=C), oracle.quantize_weight(w, pad_to=C)
+    xc, xs = to_cuda(xa["codes"]), to_cuda(xa["scale"])
+    wc, ws = to_cuda(wq["codes"]), to_cuda(wq["scale"])
+    want_acc = not bf16_out and M * O < 4_000_000
+    acc = torch.full((M, O, 1), 12345, dtype=torch.int32, device="cuda") if want_acc else None
+    wsp = tdq.linear_workspace(M, C, O, C, "cuda")
+    y = tdq.w4a4_linear(xc, xs, wc, ws, to_cuda(bias), g=C, out_dtype=torch.bfloat16 if bf16_out else torch.float32,
+                        acc_debug=acc, workspace=wsp)
+    st, detail = tdq.workspace_status(wsp)
+    assert st == tdq.OK, "device wait ran out: 0x%x" % detail
+    ref = oracle.w4a4_linear(xa["codes"], xa["scale"], wq["codes"], wq["scale"], bias=bias, g=C, want_acc=want_acc)
+    if want_acc:
+        np.testing.assert_array_equal(acc.cpu().numpy(), ref["acc"])      # the sum of the two accumulators, bit-exact
+    compare_y(y.float().cpu().numpy(), ref, 2, out_eps=2.0 ** -8 if bf16_out else 0.0)
+    # a second call on the same workspace reproduces the first bit for bit (the accumulator pairs alternate per tile)
+    y2 = tdq.w4a4_linear(xc, xs, wc, ws, to_cuda(bias), g=C, out_dtype=y.dtype, workspace=wsp)
+    assert torch.equal(y, y2)
