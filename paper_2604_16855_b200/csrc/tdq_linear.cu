@@ -294,22 +294,22 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                         // the chunks of that warp's groups (group = steps_per_grp / 4 consecutive chunks of a tile)
                         // (pair_groups == 2: one group per tile, its chunks go to the two warps in turn)
                         const int cpg = a.pair_groups == 2 ? 1 : a.steps_per_grp / kChunk;
-                        const int kc_step = a.pair_groups == 2 ? 2 : 1;
-                        for (int kc = a.pair_groups == 2 ? warp : 0; kc < n_chunks && ok; kc += kc_step) {
-                            if (a.pair_groups != 2 && ((kc / cpg) & 1) != warp) continue;
-                            const uint32_t st = 2 * ps + (uint32_t)warp;
-                            ok = mbar_wait_warp(&c->empty[st], pph ^ 1, c, a.status, 5u);
-                            if (!ok) break;
-                            if (lane == 0) {
-                                const uint32_t stage = ring_s + st * a.stage_bytes;
-                                mbar_expect_tx(&c->full[st], (uint32_t)kChunk * kBlock * (resident ? 1u : 2u));
-                                bulk_load(stage, b_src + (int64_t)kc * kChunk * kBlock, (uint32_t)kChunk * kBlock, &c->full[st]);
-                                if (!resident)
-                                    bulk_load(stage + kChunk * kBlock, a_src + (int64_t)kc * kChunk * kBlock,
-                                              (uint32_t)kChunk * kBlock, &c->full[st]);
+                        for (int kc0 = warp * cpg; kc0 < n_chunks && ok; kc0 += 2 * cpg) {
+                            for (int kc = kc0; kc < kc0 + cpg; ++kc) {
+                                const uint32_t st = 2 * ps + (uint32_t)warp;
+                                ok = mbar_wait_warp(&c->empty[st], pph ^ 1, c, a.status, 5u);
+                                if (!ok) break;
+                                if (lane == 0) {
+                                    const uint32_t stage = ring_s + st * a.stage_bytes;
+                                    mbar_expect_tx(&c->full[st], (uint32_t)kChunk * kBlock * (resident ? 1u : 2u));
+                                    bulk_load(stage, b_src + (int64_t)kc * kChunk * kBlock, (uint32_t)kChunk * kBlock, &c->full[st]);
+                                    if (!resident)
+                                        bulk_load(stage + kChunk * kBlock, a_src + (int64_t)kc * kChunk * kBlock,
+                                                  (uint32_t)kChunk * kBlock, &c->full[st]);
+                                }
+                                __syncwarp();
+                                if (++ps == n_mine) { ps = 0; pph ^= 1; }
                             }
-                            __syncwarp();
-                            if (++ps == n_mine) { ps = 0; pph ^= 1; }
                         }
                         continue;
                     }
@@ -383,7 +383,39 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                         uint32_t slot = 0;
                         bool slot_ready = false;   // the early answer about the next slot, if it was yes
                         uint32_t a_lo = ares_lo;   // resident: walks through the item's A blocks
-                        uint32_t grp = 0;          // PAIRQ: group of the tile this chunk belongs to
+                        if (PAIRQ) {
+                            // this warp's groups only (me, me + 2, ...): a group is spg / 4 consecutive chunks into slot
+                            // group & 3.  The warp has every second ring stage to itself (fed by the producer warp of the
+                            // same parity): two independent rings, so neither warp ever looks at a barrier of the other's.
+                            const int cpg = spg / kChunk;
+                            const uint32_t full_s = smem_u32(&c->full[0]);
+                            for (uint32_t g2 = me; g2 < (uint32_t)a.Kg && ok; g2 += 2) {
+                                const uint32_t gslot = g2 & (kSlots - 1), d_tmem = tmem_base + gslot * kBN;
+                                uint32_t a_g = ares_lo + g2 * (uint32_t)spg * (uint32_t)(kBlock >> 4);
+                                for (int cc = 0; cc < cpg; ++cc) {
+                                    const uint32_t st = 2 * ps + me;
+                                    if (!mbar_test_s(full_s + st * 8, pph)) {
+                                        ok = mbar_wait_warp(&c->full[st], pph, c, a.status, 4u);
+                                        if (!ok) break;
+                                    }
+                                    if (cc == 0 && !mbar_test_s(tempty_s + gslot * 8, (qm >> gslot) & 1u)) {
+                                        ok = mbar_wait_warp(&c->tempty[gslot], (qm >> gslot) & 1u, c, a.status, 3u);
+                                        if (!ok) break;
+                                    }
+                                    tc_fence_after();
+                                    const uint32_t b_st = ring_lo + st * stage_step;
+                                    mma_issue4_if<I8>(lane0, d_tmem, resident ? a_g : b_st + a_in_stage, b_st, cc == 0 ? 0u : 1u);
+                                    if (cc == cpg - 1) {
+                                        mma_commit_if(lane0, tfull_s + gslot * 8);
+                                        qm ^= 1u << gslot;
+                                    }
+                                    mma_commit_if(lane0, empty_s + st * 8);
+                                    a_g += kChunk * (kBlock >> 4);
+                                    if (++ps == n_mine) { ps = 0; pph ^= 1; }
+                                }
+                            }
+                            continue;
+                        }
                         if (SPLITQ) {
                             // this warp's chunks only (me, me + 2, ...), with as little scalar work around the four
                             // instructions as possible: a lone warp pays several clocks for every dependent instruction
@@ -416,34 +448,6 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                             continue;
                         }
                         for (int k0 = 0; k0 < n_steps && ok; k0 += kChunk) {
-                            if (PAIRQ) {
-                                // A group is spg / 4 consecutive chunks and belongs to the warp of its parity, which has
-                                // every second ring stage to itself (fed by the producer warp of the same parity): two
-                                // independent rings, so neither warp ever looks at a barrier of the other's.
-                                if ((grp & 1u) == me) {
-                                    const uint32_t st = 2 * ps + me, gslot = grp & (kSlots - 1);
-                                    ok = mbar_wait_warp(&c->full[st], pph, c, a.status, 4u);
-                                    if (!ok) break;
-                                    if (sub == 0 && !__all_sync(0xffffffffu, mbar_test_s(tempty_s + gslot * 8, (qm >> gslot) & 1u))) {
-                                        ok = mbar_wait_warp(&c->tempty[gslot], (qm >> gslot) & 1u, c, a.status, 3u);
-                                        if (!ok) break;
-                                    }
-                                    tc_fence_after();
-                                    const uint32_t b_st = ring_lo + st * stage_step;
-                                    mma_issue4_if<I8>(lane0, tmem_base + gslot * kBN, resident ? a_lo : b_st + a_in_stage, b_st,
-                                                      sub == 0 ? 0u : 1u);
-                                    if (sub + kChunk == spg) {
-                                        mma_commit_if(lane0, tfull_s + gslot * 8);
-                                        qm ^= 1u << gslot;
-                                    }
-                                    mma_commit_if(lane0, empty_s + st * 8);
-                                    if (++ps == n_mine) { ps = 0; pph ^= 1; }
-                                }
-                                sub += kChunk;
-                                if (sub == spg) { sub = 0; ++grp; }
-                                if (resident) a_lo += kChunk * (kBlock >> 4);
-                                continue;
-                            }
                             ok = mbar_wait_warp(&c->full[s], ph, c, a.status, 4u);
                             if (!ok) break;
                             const uint32_t b_lo = ring_lo + s * stage_step;
