@@ -561,9 +561,9 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
         constexpr int esz = YBF16 ? 2 : 4;
         constexpr uint32_t kRowBytes = kCols * esz;   // one row of the strip
         const uint32_t strips_s = (sm_s + a.staging_off + 1023u) & ~1023u;   // the swizzle pattern repeats every 1024 bytes
-        const bool narrow = YBF16 || a.half_strips;   // 64-byte strip rows
+        const bool narrow = YBF16 || a.half_strips;   // 64-byte strip rows (32-byte rows when a.half_strips == 2)
         const uint32_t strip_w = strips_s + (uint32_t)pw * (a.staging_bytes / kPromoWarps);
-        const uint32_t strip_row = strip_w + (uint32_t)lane * (narrow ? 64u : 128u);
+        const uint32_t strip_row = strip_w + (uint32_t)lane * (a.half_strips == 2 ? 32u : narrow ? 64u : 128u);
         const uint32_t swz = narrow ? (((uint32_t)lane >> 1) & 3u) : ((uint32_t)lane & 7u);   // chunk c sits at c ^ swz
         const uint32_t wsb_s = strips_s + a.staging_bytes + (uint32_t)pw * 256;
         uint32_t ib = 0, iu = 0;                      // item buffer and its phase
@@ -714,8 +714,62 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                 }
             }
         };
+        // The same with strip rows of 32 bytes (a.half_strips == 2: one group per tile with streamed operands, where a
+        // tile takes tens of thousands of clocks and the ring can use the shared memory): four passes of 8 columns for
+        // fp32 output, two of 16 for 16-bit output; 16 KB of strips in all.  The two 16-byte chunks of a row swap
+        // places in rows 4-7 of every eight (the 32-byte swizzle of the tensor map), which keeps the writes
+        // conflict-free.
+        auto finish_tile_quarter = [&]() {
+            float* wsb = reinterpret_cast<float*>(smem_raw + (wsb_s - sm_s));
+            wsb[lane] = __fmul_rn(w0, a.out_scale);
+            wsb[32 + lane] = b0;
+            uint8_t* strip = smem_raw + (strip_row - sm_s);
+            const uint32_t sw32 = ((uint32_t)lane >> 2) & 1u;
+            const int64_t m0 = (int64_t)mt * kBM + quarter * 32;
+            constexpr int kPasses = YBF16 ? 2 : 4, kColsPass = kCols / kPasses;
+#pragma unroll
+            for (int h = 0; h < kPasses; ++h) {
+                if (lane == 0) bulk_wait_group_read0();      // the previous pass's store has read the strip
+                __syncwarp();
+#pragma unroll
+                for (int jj = 0; jj < 2; ++jj) {             // the row's two 16-byte chunks
+                    if (YBF16) {                             // eight columns per chunk
+                        const int j = 4 * h + 2 * jj;        // yacc pairs j .. j + 3 = columns 2 j .. 2 j + 7 ... in units of four columns below
+                        float o[8];
+                        unpack2(yacc[2 * j], o[0], o[1]);
+                        unpack2(yacc[2 * j + 1], o[2], o[3]);
+                        unpack2(yacc[2 * j + 2], o[4], o[5]);
+                        unpack2(yacc[2 * j + 3], o[6], o[7]);
+                        const float4 sa = reinterpret_cast<const float4*>(wsb)[j], sb = reinterpret_cast<const float4*>(wsb)[j + 1];
+                        const float4 ba = reinterpret_cast<const float4*>(wsb + 32)[j], bb = reinterpret_cast<const float4*>(wsb + 32)[j + 1];
+                        *reinterpret_cast<uint4*>(strip + (((uint32_t)jj ^ sw32) << 4)) =
+                            make_uint4(pack16(__fmaf_rn(sa.x, o[0], ba.x), __fmaf_rn(sa.y, o[1], ba.y), a.y_f16),
+                                       pack16(__fmaf_rn(sa.z, o[2], ba.z), __fmaf_rn(sa.w, o[3], ba.w), a.y_f16),
+                                       pack16(__fmaf_rn(sb.x, o[4], bb.x), __fmaf_rn(sb.y, o[5], bb.y), a.y_f16),
+                                       pack16(__fmaf_rn(sb.z, o[6], bb.z), __fmaf_rn(sb.w, o[7], bb.w), a.y_f16));
+                    } else {                                 // four columns per chunk
+                        const int j = 2 * h + jj;
+                        float o0, o1, o2, o3;
+                        unpack2(yacc[2 * j], o0, o1);
+                        unpack2(yacc[2 * j + 1], o2, o3);
+                        const float4 s4 = reinterpret_cast<const float4*>(wsb)[j], b4 = reinterpret_cast<const float4*>(wsb + 32)[j];
+                        *reinterpret_cast<float4*>(strip + (((uint32_t)jj ^ sw32) << 4)) =
+                            make_float4(__fmaf_rn(s4.x, o0, b4.x), __fmaf_rn(s4.y, o1, b4.y), __fmaf_rn(s4.z, o2, b4.z),
+                                        __fmaf_rn(s4.w, o3, b4.w));
+                    }
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0 && m0 < a.M && n0 + kColsPass * h < a.O) {
+                    tma_store_2d(&ymap, strip_w, (int32_t)n0 + kColsPass * h, (int32_t)m0);
+                    bulk_commit_group();
+                }
+            }
+        };
         auto finish_tile = [&]() {
-            if (!YBF16 && a.half_strips) {
+            if (a.half_strips == 2) {
+                finish_tile_quarter();
+            } else if (!YBF16 && a.half_strips) {
                 finish_tile_half();
             } else {
             if (store_pending) issue_store();            // a short tile: the previous store is still waiting for its turn
@@ -1017,14 +1071,23 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
                        M <= INT32_MAX;
     const bool half_strips = y_tma && y_dtype == TDQ_F32 && !fx && !acc_debug && group_size >= 128;
     const bool narrow_strips = y_tma && (y_dtype == TDQ_BF16 || half_strips);
-    const int64_t staging_bytes = narrow_strips ? kStagingBytes / 2 : kStagingBytes;
-    if (!make_plan(M, I_pad, O, group_size, n_sm, p, staging_bytes)) return TDQ_ERR_UNSUPPORTED;
-    if (fx && !p.a_resident) return TDQ_ERR_UNSUPPORTED;   // the fused producer writes a whole row block's A into shared memory
-
-    uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
     // several instructions chain into one slot: keep the integer accumulator (the power-of-two variant
     // accumulates scaled values, which only the fp32 accumulator can hold)
     const bool i8 = group_size > 32 && !pow2_steps;
+    int64_t staging_bytes = narrow_strips ? kStagingBytes / 2 : kStagingBytes;
+    if (!make_plan(M, I_pad, O, group_size, n_sm, p, staging_bytes)) return TDQ_ERR_UNSUPPORTED;
+    // One group per tile whose operands all stream through the ring (a long contraction): the ring is what bounds the
+    // kernel there, each of the two MMA-issuing warps has half of it, and strips with 32-byte rows (16 KB in all, written
+    // in passes) leave room for a sixth stage.
+    const bool quarter_strips = y_tma && !fx && !acc_debug && i8 && p.Kg == 1 && p.n_steps % kChunk == 0 && p.n_chunks >= 2 &&
+                                !p.a_resident;
+    if (quarter_strips) {
+        staging_bytes = kStagingBytes / 4;
+        if (!make_plan(M, I_pad, O, group_size, n_sm, p, staging_bytes) || p.a_resident) return TDQ_ERR_UNSUPPORTED;
+    }
+    if (fx && !p.a_resident) return TDQ_ERR_UNSUPPORTED;   // the fused producer writes a whole row block's A into shared memory
+
+    uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
 
     ExpandArgs e;
     e.xcodes = xcodes; e.xscale = xscale; e.wcodes = wcodes;
@@ -1064,13 +1127,14 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
     a.tma_ok = 0;
     // g = 32 with y that tensor stores can write goes to the kernel built for it (tdq_linear_g32.cu)
     const bool use_g32 = !i8 && !pow2_steps && !fx && y_tma;
-    if (y_tma && encode_y_map(&ymap, y, y_dtype == TDQ_BF16, M, O, y_row_stride, half_strips ? kCols / 2 : kCols,
+    if (y_tma && encode_y_map(&ymap, y, y_dtype == TDQ_BF16, M, O, y_row_stride,
+                              quarter_strips ? (y_dtype == TDQ_BF16 ? kCols / 2 : kCols / 4) : half_strips ? kCols / 2 : kCols,
                               use_g32 ? kBM : 32, y_f16))
         a.tma_ok = 1;
-    else if (narrow_strips)
+    else if (narrow_strips || quarter_strips)
         return TDQ_ERR_CUDA;   // the plan counted on the tensor store
     a.staging_bytes = (uint32_t)staging_bytes;
-    a.half_strips = half_strips ? 1 : 0;
+    a.half_strips = quarter_strips ? 2 : half_strips ? 1 : 0;
     a.out_scale = i8 ? 0.00390625f : 262144.0f;
     a.y_f16 = y_f16 ? 1 : 0;
     a.xcodes = xcodes; a.xscale = xscale; a.row_bytes = e.row_bytes; a.unpack_a = unpack_a ? 1 : 0;

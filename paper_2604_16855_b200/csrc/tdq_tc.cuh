@@ -56,8 +56,9 @@ struct LinArgs {
     int32_t a_resident;        // the item's whole A block stays in shared memory
     int32_t n_stages;
     uint32_t ring_off, stage_bytes, staging_off;   // shared-memory carve-up
-    uint32_t staging_bytes;    // all sixteen strips: 64 KB, or 32 KB when a strip holds 32 rows of 64 bytes
-    int32_t half_strips;       // fp32 output written in two passes of 16 columns through 64-byte strip rows
+    uint32_t staging_bytes;    // all sixteen strips: 64 KB, 32 KB when a strip holds 32 rows of 64 bytes, 16 KB with rows of 32 bytes
+    int32_t half_strips;       // 1: fp32 output written in two passes of 16 columns through 64-byte strip rows; 2: any output in
+                               // passes through 32-byte strip rows
     uint32_t ibuf_bytes;       // one item buffer: the item's scales, then its A blocks if resident
     int32_t n_ibuf;            // item buffers (1..kMaxItemBufs): the producer runs that many items ahead
     void* y;
@@ -412,10 +413,10 @@ bool encode_y_map(CUtensorMap* map, void* y, bool bf16, int64_t M, int64_t O, in
     const cuuint64_t dims[2] = {(cuuint64_t)O, (cuuint64_t)M};
     const cuuint64_t strides[1] = {(cuuint64_t)y_row_stride * esz};
     const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
-    const bool rows64 = (size_t)box_cols * esz == 64;   // 64-byte strip rows (else 128)
+    const size_t row_bytes = (size_t)box_cols * esz;    // strip rows of 128, 64 or 32 bytes, swizzled alike
     const cuuint32_t elem_strides[2] = {1u, 1u};
     return encode(map, bf16 ? (f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16) : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, y, dims, strides, box,
-                  elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, rows64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                  elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, row_bytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
                   CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
