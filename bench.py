@@ -725,9 +725,15 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="only the timed steps, the per-kernel timings and the end-to-end leg (for profiler runs)")
     ap.add_argument("--oracle-leg", type=int, default=0, help=argparse.SUPPRESS)
     ap.add_argument("--eager", action="store_true", help="launch every timed step from the host instead of replaying a CUDA graph")
+    ap.add_argument("--probe-only", action="store_true", help="only the compute-bound probe shape of the linear layer (for profiler runs); prints that leg")
     args = ap.parse_args()
     if args.oracle_leg:                    # child of cpu_oracle_single_thread
         print(json.dumps(cpu_oracle_leg(workload(args.workload), args.oracle_leg)))
+        return
+    if args.probe_only:
+        import torch
+        from paper_2604_16855_b200 import tdq
+        print(json.dumps(dict(compute_probe=probe_leg(tdq, torch.device("cuda", 0), load_peaks()))))
         return
     if args.steps is None:
         args.steps = 10 if args.impl == "reference" else 1000
