@@ -34,8 +34,12 @@
 //        warps 2-3   MMA issue and the commits that release buffers.  Group k of a tile uses TMEM slot
 //                    k & 3.  The issue loop is straight-line, predicated code (a lone warp runs
 //                    dependent scalar code slowly, and branches cost most): at g = 32 the two warps take
-//                    the even and the odd slots, at g = 64 the first and the second group of a stage,
-//                    at g a multiple of 128 warp 2 issues a stage's four steps in a row.
+//                    the even and the odd slots, at g = 64 the first and the second group of a stage.
+//                    At g a multiple of 128 a ring stage belongs to one group: with two or more groups per
+//                    tile the two warps take the groups in turn, with one group per tile (g = C) they take
+//                    its stages in turn, each into an accumulator of its own that the promotion warps add
+//                    (integer sums); either way each warp has its own half of the ring, fed by the
+//                    producer warp of its parity.  Otherwise warp 2 issues alone.
 //        warps 4-19  promotion + epilogue: warp w owns TMEM lanes 32 (w % 4).. (its rows) and 32
 //                    columns; a thread keeps 32 float accumulators of one output row and one
 //                    32-value landing buffer.  Sixteen warps, four per scheduler: a warp executes
@@ -51,6 +55,8 @@
 //      bulk tensor store; lane 0 starts one 32 x 32 store per tile, a few groups into the next
 //      tile, and the copy engine clips it at the edges of y.  Unaligned y is written element by
 //      element from the same strip.
+//      Where the ring needs the shared memory more (wide groups), the strips have rows of 64 or 32 bytes
+//      and a tile is written in two or four passes.
 //   The fused instantiation (tdq_quant_linear_fused) replaces the load of an item's A block and
 //   scales: the promotion warps quantize the item's 128 activation rows into the same shared-memory
 //   regions before they start on its tiles.
