@@ -443,10 +443,11 @@ bool make_plan(int64_t M, int64_t I_pad, int64_t O, int32_t g, int n_sm, Plan& p
     if (stages_res >= 3) {
         p.a_resident = 1;
         p.ibuf_bytes = (uint32_t)(scales + a_res);
-        // further item buffers while at least six stages remain: with short contractions the hand-over
-        // between work items, not the ring, is what the tensor core waits for
+        // further item buffers while enough stages remain for two tiles' worth of B (at most six, at least three):
+        // with short contractions the hand-over between work items, not the ring, is what the tensor core waits for
+        const int64_t want_stages = 2 * p.n_chunks < 3 ? 3 : (2 * p.n_chunks > 6 ? 6 : 2 * p.n_chunks);
         p.n_ibuf = 1;
-        while (p.n_ibuf < kMaxItemBufs && (kSmemLimit - fixed - a_res - (int64_t)p.n_ibuf * p.ibuf_bytes) / stage_b >= 6) ++p.n_ibuf;
+        while (p.n_ibuf < kMaxItemBufs && (kSmemLimit - fixed - a_res - (int64_t)p.n_ibuf * p.ibuf_bytes) / stage_b >= want_stages) ++p.n_ibuf;
         const int64_t st = (kSmemLimit - fixed - a_res - (int64_t)(p.n_ibuf - 1) * p.ibuf_bytes) / stage_b;
         p.n_stages = (int32_t)(st > kMaxStages ? kMaxStages : st);
         p.stage_bytes = (uint32_t)stage_b;
