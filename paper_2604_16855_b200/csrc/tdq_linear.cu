@@ -295,7 +295,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                 if (++ib == (uint32_t)a.n_ibuf) { ib = 0; iu ^= 1; }
                 for (int nt = part_begin(part); nt < part_begin(part + 1) && ok; ++nt) {
                     const uint8_t* b_src = a.b_blocks + (int64_t)nt * a.n_steps * kBlock;
-                    if (I8 && a.pair_groups) {   // (wide groups always take the integer instruction)
+                    if (!FUSED && a.pair_groups) {   // (not compiled into the fused kernels, which never take these modes)
                         // two rings: this warp feeds the MMA warp of its parity through the stages of its parity, with
                         // the chunks of that warp's groups (group = steps_per_grp / 4 consecutive chunks of a tile)
                         // (pair_groups == 2: one group per tile, its chunks go to the two warps in turn)
@@ -338,7 +338,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                     }
                 }
             }
-        } else if (warp == kMmaWarp || spg <= 2 || (I8 && a.pair_groups)) {
+        } else if (warp == kMmaWarp || spg <= 2 || (!FUSED && a.pair_groups)) {
             // ------------------------------------------------------------ MMA issue (lane 0 issues)
             // A warp runs dependent scalar code at one instruction every few clocks, so this loop is
             // what paces the tensor pipe: everything that can be is hoisted, and the two cases are
@@ -545,7 +545,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
             };
             if (spg == 1) role(std::integral_constant<int, 0>{});
             else if (spg == 2) role(std::integral_constant<int, 3>{});
-            else if (I8 && a.pair_groups == 2) role(std::integral_constant<int, 5>{});
+            else if (!FUSED && a.pair_groups == 2) role(std::integral_constant<int, 5>{});
             else if (I8 && a.pair_groups) role(std::integral_constant<int, 4>{});
             else if (spg % kChunk == 0) role(std::integral_constant<int, 1>{});
             else role(std::integral_constant<int, 2>{});
@@ -890,7 +890,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
             return next_ready;
         };
         // One group per tile in two accumulators (a.pair_groups == 2): slots UA and UA + 1 hold the sums over the even
-        // and the odd chunks of K.  Integer sums: their sum is the group's sum whatever the split.
+        // and the odd chunks of K.  Integer sums: their sum is the group's sum whatever the split.  (The power-of-two
+        // variant accumulates scaled values in fp32; there the split adds one rounding to the K the variant already has.)
         auto consume_split = [&](auto u_tag) {
             constexpr uint32_t UA = decltype(u_tag)::value, UB = UA + 1;
             ok = mbar_wait_warp(&c->tfull[UA], p_full[UA], c, a.status, 2u);
@@ -912,7 +913,11 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
                     tmem_ld16(tmem_row_r + UB * kBN + h * (kCols / 2), v2);
                     tmem_ld_wait_on16(v2);
 #pragma unroll
-                    for (int q = 0; q < kCols / 2; ++q) v[h * (kCols / 2) + q] += v2[q];
+                    for (int q = 0; q < kCols / 2; ++q) {
+                        uint32_t& d = v[h * (kCols / 2) + q];
+                        if (I8) d += v2[q];
+                        else d = __float_as_uint(__fadd_rn(__uint_as_float(d), __uint_as_float(v2[q])));   // power-of-two variant
+                    }
                 }
             }
             tc_fence_before();                            // both slots are drained
@@ -925,7 +930,8 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
             }
             if (!FUSED) {
 #pragma unroll
-                for (int q = 0; q < kCols; ++q) v[q] = __float_as_uint((float)(int32_t)v[q]);
+                for (int q = 0; q < kCols; ++q)
+                    if (I8) v[q] = __float_as_uint((float)(int32_t)v[q]);
 #pragma unroll
                 for (int q = 0; q < kCols / 2; ++q) fma2(yacc[q], pack2(v[2 * q], v[2 * q + 1]), d2);
             }
@@ -935,7 +941,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
         const std::integral_constant<uint32_t, 2> u2{};
         const std::integral_constant<uint32_t, 3> u3{};
 
-        if (I8 && !FUSED && a.pair_groups == 2) {
+        if (!FUSED && a.pair_groups == 2) {
             if (item < n_items) {
                 begin_item();
                 if (ok) begin_tile();
@@ -1085,7 +1091,7 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
     // One group per tile whose operands all stream through the ring (a long contraction): the ring is what bounds the
     // kernel there, each of the two MMA-issuing warps has half of it, and strips with 32-byte rows (16 KB in all, written
     // in passes) leave room for a sixth stage.
-    const bool quarter_strips = y_tma && !fx && !acc_debug && i8 && p.Kg == 1 && p.n_steps % kChunk == 0 && p.n_chunks >= 2 &&
+    const bool quarter_strips = y_tma && !fx && !acc_debug && (i8 || pow2_steps) && p.Kg == 1 && p.n_steps % kChunk == 0 && p.n_chunks >= 2 &&
                                 !p.a_resident;
     if (quarter_strips) {
         staging_bytes = kStagingBytes / 4;
@@ -1146,7 +1152,7 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
     a.xcodes = xcodes; a.xscale = xscale; a.row_bytes = e.row_bytes; a.unpack_a = unpack_a ? 1 : 0;
     a.pair_groups = (i8 && a.steps_per_grp % kChunk == 0 && a.Kg >= 2) ? 1 : 0;
     // one group per tile: the group's chunks go to the two MMA warps in turn, each with an accumulator of its own
-    if (i8 && !fx && a.Kg == 1 && a.steps_per_grp % kChunk == 0 && p.n_chunks >= 2) a.pair_groups = 2;
+    if ((i8 || pow2_steps) && !fx && a.Kg == 1 && a.steps_per_grp % kChunk == 0 && p.n_chunks >= 2) a.pair_groups = 2;
     a.x = fx ? fx->x : nullptr;
     a.x_stride = fx ? fx->row_stride : 0;
     a.seven_tau = fx ? fx->seven_tau : 0.0f;
