@@ -1091,11 +1091,17 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
     // One group per tile whose operands all stream through the ring (a long contraction): the ring is what bounds the
     // kernel there, each of the two MMA-issuing warps has half of it, and strips with 32-byte rows (16 KB in all, written
     // in passes) leave room for a sixth stage.
-    const bool quarter_strips = y_tma && !fx && !acc_debug && (i8 || pow2_steps) && p.Kg == 1 && p.n_steps % kChunk == 0 && p.n_chunks >= 2 &&
-                                !p.a_resident;
+    bool quarter_strips = y_tma && !fx && !acc_debug && (i8 || pow2_steps) && p.Kg == 1 && p.n_steps % kChunk == 0 && p.n_chunks >= 2 &&
+                          !p.a_resident;
     if (quarter_strips) {
-        staging_bytes = kStagingBytes / 4;
-        if (!make_plan(M, I_pad, O, group_size, n_sm, p, staging_bytes) || p.a_resident) return TDQ_ERR_UNSUPPORTED;
+        // (with the smaller strips A may fit after all; that case keeps the plan it had)
+        Plan q;
+        if (make_plan(M, I_pad, O, group_size, n_sm, q, kStagingBytes / 4) && !q.a_resident) {
+            p = q;
+            staging_bytes = kStagingBytes / 4;
+        } else {
+            quarter_strips = false;
+        }
     }
     if (fx && !p.a_resident) return TDQ_ERR_UNSUPPORTED;   // the fused producer writes a whole row block's A into shared memory
 

@@ -307,7 +307,9 @@ def test_fp16_output(tdq, idx, rows, g, fused):
 @pytest.mark.parametrize("M,C,O,bf16_out", [(300, 256, 200, False), (20000, 384, 384, False), (700, 640, 130, True),
                                             (2100, 768, 1280, False), (129, 1024, 700, True), (5000, 128, 96, False),
                                             # operands streamed (K too long to stay resident): strips with 32-byte rows, written in passes
-                                            (300, 2048, 200, False), (260, 4096, 130, True), (700, 2176, 100, False), (40000, 2048, 128, True)])
+                                            (300, 2048, 200, False), (260, 4096, 130, True), (700, 2176, 100, False), (40000, 2048, 128, True),
+                                            # K at which the operands stream with the usual strips but would stay resident with the small ones
+                                            (300, 1152, 200, False), (2500, 1152, 64, True)])
 def test_one_group_per_token_split_over_two_accumulators(tdq, M, C, O, bf16_out):
     rng = np.random.RandomState(M + 3 * C + O)
     x = (rng.normal(size=(M, C)) * np.exp(rng.normal(0, 1.0, size=(M, 1)))).astype(np.float32)
