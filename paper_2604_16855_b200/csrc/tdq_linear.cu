@@ -1091,12 +1091,14 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
     // One group per tile whose operands all stream through the ring (a long contraction): the ring is what bounds the
     // kernel there, each of the two MMA-issuing warps has half of it, and strips with 32-byte rows (16 KB in all, written
     // in passes) leave room for a sixth stage.
-    bool quarter_strips = y_tma && !fx && !acc_debug && (i8 || pow2_steps) && p.Kg == 1 && p.n_steps % kChunk == 0 && p.n_chunks >= 2 &&
-                          !p.a_resident;
+    // One group per tile: the ring is what bounds the kernel there, each of the two MMA-issuing warps has half of it, and
+    // strips with 32-byte rows (16 KB in all, written in passes) leave room for more stages.  Taken when that gives the
+    // smaller half of the ring another stage without changing whether A stays resident.
+    bool quarter_strips = y_tma && !fx && !acc_debug && (i8 || pow2_steps) && p.Kg == 1 && p.n_steps % kChunk == 0 && p.n_chunks >= 2;
     if (quarter_strips) {
-        // (with the smaller strips A may fit after all; that case keeps the plan it had)
         Plan q;
-        if (make_plan(M, I_pad, O, group_size, n_sm, q, kStagingBytes / 4) && !q.a_resident) {
+        if (make_plan(M, I_pad, O, group_size, n_sm, q, kStagingBytes / 4) && q.a_resident == p.a_resident &&
+            q.n_stages / 2 > p.n_stages / 2) {
             p = q;
             staging_bytes = kStagingBytes / 4;
         } else {
