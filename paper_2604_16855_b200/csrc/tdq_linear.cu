@@ -1088,13 +1088,13 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
     const bool i8 = group_size > 32 && !pow2_steps;
     int64_t staging_bytes = narrow_strips ? kStagingBytes / 2 : kStagingBytes;
     if (!make_plan(M, I_pad, O, group_size, n_sm, p, staging_bytes)) return TDQ_ERR_UNSUPPORTED;
-    // One group per tile whose operands all stream through the ring (a long contraction): the ring is what bounds the
-    // kernel there, each of the two MMA-issuing warps has half of it, and strips with 32-byte rows (16 KB in all, written
-    // in passes) leave room for a sixth stage.
-    // One group per tile: the ring is what bounds the kernel there, each of the two MMA-issuing warps has half of it, and
-    // strips with 32-byte rows (16 KB in all, written in passes) leave room for more stages.  Taken when that gives the
-    // smaller half of the ring another stage without changing whether A stays resident.
-    bool quarter_strips = y_tma && !fx && !acc_debug && (i8 || pow2_steps) && p.Kg == 1 && p.n_steps % kChunk == 0 && p.n_chunks >= 2;
+    // Wide groups run with two MMA-issuing warps, each with half of the ring, and the ring is what bounds them: strips
+    // with 32-byte rows (16 KB in all, written in passes) leave room for more stages.  Taken when that gives the smaller
+    // half of the ring another stage without changing whether A stays resident; with several groups per tile only where
+    // the operands stream (a long contraction), since the passes cost a short tile more than the stage gives.
+    bool quarter_strips = y_tma && !fx && !acc_debug && (i8 || pow2_steps) && p.n_chunks >= 2 &&
+                          ((p.Kg == 1 && p.n_steps % kChunk == 0) ||
+                           (i8 && (group_size / 32) % kChunk == 0 && p.Kg >= 2 && !p.a_resident));
     if (quarter_strips) {
         Plan q;
         if (make_plan(M, I_pad, O, group_size, n_sm, q, kStagingBytes / 4) && q.a_resident == p.a_resident &&
