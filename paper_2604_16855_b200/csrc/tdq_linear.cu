@@ -64,6 +64,8 @@
 // Every wait on an mbarrier is bounded: after about a second the thread records a code in the
 // workspace status word and raises a CTA-wide flag; every role then leaves its loops, the CTA
 // releases its TMEM and returns.
+#include <cuda_fp8.h>
+
 #include <mutex>
 
 #include "tdq_act_group.cuh"
@@ -138,18 +140,18 @@ __global__ void __launch_bounds__(kExpandThreads) expand_kernel(ExpandArgs a) {
 // the byte is exact.  Steps more than 2^14 below the row's largest have s < 0 and lose their low bits
 // (truncated).  The whole contraction then accumulates in one fp32 accumulator and the row needs one
 // scale, 2^e_m, in the epilogue.
-__device__ __forceinline__ uint32_t pow2_byte(uint32_t nib, int s) {
-    const uint32_t neg = nib & 8u;
-    const uint32_t mag = neg ? 16u - nib : nib;            // |q| in 0..8
-    const uint32_t t = s >= 0 ? mag << s : mag >> min(-s, 31);
-    uint32_t b;
-    if (t < 8u) {
-        b = t;                                             // subnormal: t * 2^-9
-    } else {
-        const int p = 31 - __clz(t);                       // t = 1.m * 2^p
-        b = ((uint32_t)(p - 2) << 3) | ((t >> (p - 3)) & 7u);
+// Four codes (the nibbles of h, lowest first) as four such bytes.  shr = max(-s, 0) low bits of |q| are dropped first;
+// mul = 2^(max(s, 0) - 9).  q * mul is exact in binary32 and in E4M3, so the hardware conversion is exact too.
+__device__ __forceinline__ uint32_t pow2_bytes4(uint32_t h, int shr, float mul) {
+    int q[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        q[i] = ((int)(h << (28 - 4 * i))) >> 28;           // sign-extended nibble
+        if (shr) q[i] = q[i] >= 0 ? (q[i] >> shr) : -((-q[i]) >> shr);   // toward zero
     }
-    return b | (neg << 4);                                 // sign bit 7
+    const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2((float)q[0] * mul, (float)q[1] * mul), __NV_SATFINITE, __NV_E4M3);
+    const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2((float)q[2] * mul, (float)q[3] * mul), __NV_SATFINITE, __NV_E4M3);
+    return lo | (hi << 16);
 }
 
 __global__ void __launch_bounds__(kExpandThreads) expand_pow2_kernel(ExpandArgs a, int32_t act_steps_per_grp, int32_t act_Kg) {
@@ -178,7 +180,16 @@ __global__ void __launch_bounds__(kExpandThreads) expand_pow2_kernel(ExpandArgs 
         if (row < rows) {
             const float* sc = a.xscale + row * act_Kg;
             uint32_t emax = 0u, bad = 0u;
-            for (int k = 0; k < act_Kg; ++k) {
+            int k = 0;
+            if ((act_Kg & 3) == 0 && (reinterpret_cast<uintptr_t>(sc) & 15) == 0) {   // four steps per load
+#pragma unroll 2
+                for (; k < act_Kg; k += 4) {
+                    const uint4 b4 = __ldg(reinterpret_cast<const uint4*>(sc + k));
+                    emax = max(max(emax, b4.x >> 23), max(max(b4.y >> 23, b4.z >> 23), b4.w >> 23));
+                    bad |= (b4.x | b4.y | b4.z | b4.w) & 0x807fffffu;
+                }
+            }
+            for (; k < act_Kg; ++k) {
                 const uint32_t bits = __float_as_uint(__ldg(sc + k));
                 emax = max(emax, bits >> 23);
                 bad |= bits & 0x807fffffu;                 // a mantissa or a sign: not a power of two
@@ -190,12 +201,11 @@ __global__ void __launch_bounds__(kExpandThreads) expand_pow2_kernel(ExpandArgs 
         }
         uint32_t w[8];
         const uint32_t pw[4] = {p.x, p.y, p.z, p.w};
+        const int shr = s < 0 ? min(-s, 31) : 0;
+        const float mul = __uint_as_float((uint32_t)((s > 0 ? s : 0) - 9 + 127) << 23);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {                      // four nibbles -> four bytes
-            const uint32_t h = (pw[i >> 1] >> (16 * (i & 1))) & 0xffffu;
-            w[i] = pow2_byte(h & 15u, s) | (pow2_byte((h >> 4) & 15u, s) << 8) | (pow2_byte((h >> 8) & 15u, s) << 16) |
-                   (pow2_byte(h >> 12, s) << 24);
-        }
+        for (int i = 0; i < 8; ++i)                        // four nibbles -> four bytes
+            w[i] = pow2_bytes4((pw[i >> 1] >> (16 * (i & 1))) & 0xffffu, shr, mul);
         c0 = make_uint4(w[0], w[1], w[2], w[3]);
         c1 = make_uint4(w[4], w[5], w[6], w[7]);
         if (ks == 0) reinterpret_cast<uint32_t*>(a.s_blocks + (int64_t)tile * kScaleBlock)[r] = row_scale;
