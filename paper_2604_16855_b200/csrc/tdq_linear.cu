@@ -1095,7 +1095,7 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
     const bool narrow_strips = y_tma && (y_dtype == TDQ_BF16 || half_strips);
     // several instructions chain into one slot: keep the integer accumulator (the power-of-two variant
     // accumulates scaled values, which only the fp32 accumulator can hold)
-    const bool i8 = group_size > 32 && !pow2_steps;
+    const bool i8 = group_size > 64 && !pow2_steps;
     int64_t staging_bytes = narrow_strips ? kStagingBytes / 2 : kStagingBytes;
     if (!make_plan(M, I_pad, O, group_size, n_sm, p, staging_bytes)) return TDQ_ERR_UNSUPPORTED;
     // Wide groups run with two MMA-issuing warps, each with half of the ring, and the ring is what bounds them: strips
@@ -1156,7 +1156,7 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
     memset(&ymap, 0, sizeof(ymap));
     a.tma_ok = 0;
     // g = 32 with y that tensor stores can write goes to the kernel built for it (tdq_linear_g32.cu)
-    const bool use_g32 = !i8 && !pow2_steps && !fx && y_tma;
+    const bool use_g32 = group_size == 32 && !pow2_steps && !fx && y_tma;
     if (y_tma && encode_y_map(&ymap, y, y_dtype == TDQ_BF16, M, O, y_row_stride,
                               quarter_strips ? (y_dtype == TDQ_BF16 ? kCols / 2 : kCols / 4) : half_strips ? kCols / 2 : kCols,
                               use_g32 ? kBM : 32, y_f16))
