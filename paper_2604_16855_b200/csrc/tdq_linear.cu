@@ -11,13 +11,14 @@
 // 128 x 128 x 32 instruction takes 64 clocks, while 16384 fp32 FMAs take 128 clocks of the SM's
 // FMA pipes.  The operand encoding is chosen so that nothing else is added to that:
 //
-//   * g = 32: kind::f8f6f4, E4M3 operands, fp32 accumulator.  A code q in [-8, 8] is stored as
+//   * g <= 128: kind::f8f6f4, E4M3 operands, fp32 accumulator.  A code q in [-8, 8] is stored as
 //     the byte sign(q) << 7 | |q|, which E4M3 reads as q * 2^-9 (the values are subnormal, or
-//     2^-6 for |q| = 8).  One instruction contracts one group into a fresh slot; the 32
-//     products (|p| <= 64) and their sum (<= 1792) are exact in the fp32 accumulator, so TMEM
-//     holds acc * 2^-18 exactly and the promotion needs no integer-to-float conversion: one
-//     packed fp32 FMA per two values.
-//   * g > 32: kind::i8, int32 accumulator (several instructions chain into one slot, so the
+//     2^-6 for |q| = 8).  g / 32 instructions contract one group into a fresh slot; the products
+//     (|p| <= 64) and their sum (<= 8192) are exact in the fp32 accumulator, so TMEM holds
+//     acc * 2^-18 exactly and the promotion needs no integer-to-float conversion: one packed fp32
+//     FMA per two values.  (Measured with adversarial codes: the accumulator stays exact up to the
+//     largest sum 4096 codes can produce, 2^18; the limit of 128 is caution, not need.)
+//   * g > 128: kind::i8, int32 accumulator (many instructions chain into one slot, so the
 //     sum stays in integers; promotion is rarer).  A code is stored as the two's complement
 //     byte 16 q; TMEM holds 256 acc.
 //   The power of two is folded into the output-channel scale in the epilogue; both routes
@@ -556,7 +557,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
             if (spg == 1) role(std::integral_constant<int, 0>{});
             else if (spg == 2) role(std::integral_constant<int, 3>{});
             else if (!FUSED && a.pair_groups == 2) role(std::integral_constant<int, 5>{});
-            else if (I8 && a.pair_groups) role(std::integral_constant<int, 4>{});
+            else if (!FUSED && a.pair_groups) role(std::integral_constant<int, 4>{});
             else if (spg % kChunk == 0) role(std::integral_constant<int, 1>{});
             else role(std::integral_constant<int, 2>{});
         }
@@ -1095,16 +1096,20 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
     const bool narrow_strips = y_tma && (y_dtype == TDQ_BF16 || half_strips);
     // several instructions chain into one slot: keep the integer accumulator (the power-of-two variant
     // accumulates scaled values, which only the fp32 accumulator can hold)
-    const bool i8 = group_size > 64 && !pow2_steps;
+    const bool wide = group_size > 64 && !pow2_steps;   // a ring stage belongs to one group: the two-warp modes
+    // Up to 128 codes per group the E4M3 route is taken (at most four chained instructions per accumulator; the sums, below
+    // 2^13 in units of 2^-18, are exact in the fp32 accumulator, and the promotion needs no integer-to-float conversion);
+    // wider groups keep the integer accumulator.
+    const bool i8 = group_size > 128 && !pow2_steps;
     int64_t staging_bytes = narrow_strips ? kStagingBytes / 2 : kStagingBytes;
     if (!make_plan(M, I_pad, O, group_size, n_sm, p, staging_bytes)) return TDQ_ERR_UNSUPPORTED;
     // Wide groups run with two MMA-issuing warps, each with half of the ring, and the ring is what bounds them: strips
     // with 32-byte rows (16 KB in all, written in passes) leave room for more stages.  Taken when that gives the smaller
     // half of the ring another stage without changing whether A stays resident; with several groups per tile only where
     // the operands stream (a long contraction), since the passes cost a short tile more than the stage gives.
-    bool quarter_strips = y_tma && !fx && !acc_debug && (i8 || pow2_steps) && p.n_chunks >= 2 &&
+    bool quarter_strips = y_tma && !fx && !acc_debug && (wide || pow2_steps) && p.n_chunks >= 2 &&
                           ((p.Kg == 1 && p.n_steps % kChunk == 0) ||
-                           (i8 && (group_size / 32) % kChunk == 0 && p.Kg >= 2 && !p.a_resident));
+                           (wide && (group_size / 32) % kChunk == 0 && p.Kg >= 2 && !p.a_resident));
     if (quarter_strips) {
         Plan q;
         if (make_plan(M, I_pad, O, group_size, n_sm, q, kStagingBytes / 4) && q.a_resident == p.a_resident &&
@@ -1168,9 +1173,9 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
     a.out_scale = i8 ? 0.00390625f : 262144.0f;
     a.y_f16 = y_f16 ? 1 : 0;
     a.xcodes = xcodes; a.xscale = xscale; a.row_bytes = e.row_bytes; a.unpack_a = unpack_a ? 1 : 0;
-    a.pair_groups = (i8 && a.steps_per_grp % kChunk == 0 && a.Kg >= 2) ? 1 : 0;
+    a.pair_groups = (wide && a.steps_per_grp % kChunk == 0 && a.Kg >= 2) ? 1 : 0;
     // one group per tile: the group's chunks go to the two MMA warps in turn, each with an accumulator of its own
-    if ((i8 || pow2_steps) && !fx && a.Kg == 1 && a.steps_per_grp % kChunk == 0 && p.n_chunks >= 2) a.pair_groups = 2;
+    if ((wide || pow2_steps) && !fx && a.Kg == 1 && a.steps_per_grp % kChunk == 0 && p.n_chunks >= 2) a.pair_groups = 2;
     a.x = fx ? fx->x : nullptr;
     a.x_stride = fx ? fx->row_stride : 0;
     a.seven_tau = fx ? fx->seven_tau : 0.0f;

@@ -332,3 +332,42 @@ def test_one_group_per_token_split_over_two_accumulators(tdq, M, C, O, bf16_out)
     # a second call on the same workspace reproduces the first bit for bit (the accumulator pairs alternate per tile)
     y2 = tdq.w4a4_linear(xc, xs, wc, ws, to_cuda(bias), g=C, out_dtype=y.dtype, workspace=wsp)
     assert torch.equal(y, y2)
+
+
+# ---------------------------------------------------------------------------------------
+# Exactness of the accumulators on constructed codes: the largest sums a group can produce and sums with busy
+# low bits (a constant operand against varied codes), on both operand routes (E4M3 with an fp32 accumulator up
+# to 128 codes per group, int8 with an int32 accumulator beyond), resident and streamed operands.
+
+def _pack_codes(q):
+    u = (q.astype(np.int16) & 15).astype(np.uint8)
+    return (u[:, 0::2] | (u[:, 1::2] << 4)).astype(np.uint8)
+
+
+@pytest.mark.parametrize("M,C,O,g", [(200, 256, 130, 32), (200, 512, 130, 64), (130, 1024, 100, 128), (130, 4096, 128, 128),
+                                     (128, 1024, 128, 256), (150, 768, 96, 768), (140, 4096, 128, 4096)])
+def test_group_sums_are_exact_on_extreme_codes(tdq, M, C, O, g):
+    rng = np.random.RandomState(g + C)
+    for kind in ("all -8", "all 7", "7 against varied", "alternating 7 / -8", "random"):
+        if kind == "all -8":
+            qx, qw = np.full((M, C), -8, np.int8), np.full((O, C), -8, np.int8)
+        elif kind == "all 7":
+            qx, qw = np.full((M, C), 7, np.int8), np.full((O, C), 7, np.int8)
+        elif kind == "7 against varied":
+            qx, qw = np.full((M, C), 7, np.int8), rng.randint(1, 8, size=(O, C)).astype(np.int8)
+        elif kind == "alternating 7 / -8":
+            qx = np.where(np.arange(C)[None, :] % 2 == 0, 7, -8).astype(np.int8).repeat(M, 0)
+            qw = rng.randint(-8, 8, size=(O, C)).astype(np.int8)
+        else:
+            qx, qw = rng.randint(-8, 8, size=(M, C)).astype(np.int8), rng.randint(-8, 8, size=(O, C)).astype(np.int8)
+        xs = np.ones((M, C // g), np.float32)
+        ws = np.ones((O,), np.float32)
+        acc = torch.full((M, O, C // g), 12345, dtype=torch.int32, device="cuda")
+        wsp = tdq.linear_workspace(M, C, O, g, "cuda")
+        y = tdq.w4a4_linear(to_cuda(_pack_codes(qx)), to_cuda(xs), to_cuda(_pack_codes(qw)), to_cuda(ws), g=g, acc_debug=acc, workspace=wsp)
+        st, detail = tdq.workspace_status(wsp)
+        assert st == tdq.OK, "device wait ran out: 0x%x" % detail
+        ref = np.einsum("mkg,okg->mok", qx.reshape(M, C // g, g).astype(np.int64), qw.reshape(O, C // g, g).astype(np.int64))
+        np.testing.assert_array_equal(acc.cpu().numpy().astype(np.int64), ref, err_msg=kind)
+        # unit steps and unit channel scales: y is the integer sum over the groups, exact in binary32 below 2^24
+        np.testing.assert_array_equal(y.cpu().numpy().astype(np.int64), ref.sum(axis=2), err_msg=kind)
