@@ -102,8 +102,7 @@ __device__ __forceinline__ void tmem_ld_wait_on16(uint32_t* v) {
 // One CTA rewrites one (128-row block, 4 K-steps) piece: thread t takes row t / 4 and K-step t % 4.
 template <bool I8>
 __global__ void __launch_bounds__(kExpandThreads) expand_kernel(ExpandArgs a) {
-    pdl_wait();
-    pdl_trigger();
+    pdl_trigger();                                         // the GEMM may set itself up meanwhile
     const int piece = blockIdx.x;
     if (piece == 0 && threadIdx.x < 4) a.status[threadIdx.x] = 0u;   // saves a separate memset in front of every call
     const int blk = piece / a.n_chunks, kc = piece % a.n_chunks;
@@ -155,66 +154,122 @@ __device__ __forceinline__ uint32_t pow2_bytes4(uint32_t h, int shr, float mul) 
     return lo | (hi << 16);
 }
 
+// Eight codes (the nibbles of p, lowest first) through a 16-entry byte table held in four registers (entry n
+// is the byte of the code whose two's-complement nibble is n): one byte permute per four codes and table half,
+// and a select on the nibble's top bit.
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+__device__ __forceinline__ void table_bytes8(uint32_t p, const uint4& tab, uint32_t& lo, uint32_t& hi) {
+    const uint32_t sel = p & 0x77777777u;                  // selectors 0..7; only the low 16 bits of a selector count
+    const uint32_t ev = (p << 4) & 0x80808080u;            // top bits of nibbles 0, 2, 4, 6 as byte signs
+    const uint32_t od = p & 0x80808080u;                   // of nibbles 1, 3, 5, 7
+    const uint32_t m_lo = prmt(ev, od, 0xd9c8u);           // sign-replicating selectors: 0xff where the nibble is >= 8
+    const uint32_t m_hi = prmt(ev, od, 0xfbeau);
+    const uint32_t a_lo = prmt(tab.x, tab.y, sel), b_lo = prmt(tab.z, tab.w, sel);
+    const uint32_t a_hi = prmt(tab.x, tab.y, sel >> 16), b_hi = prmt(tab.z, tab.w, sel >> 16);
+    lo = (a_lo & ~m_lo) | (b_lo & m_lo);
+    hi = (a_hi & ~m_hi) | (b_hi & m_hi);
+}
+
+constexpr int kPow2MinShift = -4;                          // |q| <= 8: four or more dropped bits leave nothing
+constexpr int kPow2Tables = 14 - kPow2MinShift + 1;        // one table per s in -4..14
+constexpr int kPow2Chunks = 2;                             // chunks of K-steps per CTA of the expansion
+
+// A step that is not a positive power of two is reported as the status word 11 | epoch << 8, stored by
+// whichever thread meets one.  The epoch is the workspace's third status word: the GEMM kernel of every call
+// adds one to it, after this kernel has finished, so it is fixed while this kernel runs and differs from the
+// epoch of the call before (also when the calls are replays of one captured graph).  The CTA that clears the
+// status word for this call leaves exactly the value 11 | epoch << 8 alone, so the order of the clear and the
+// reports does not matter, and a report left by an earlier call is cleared like any other stale word.
 __global__ void __launch_bounds__(kExpandThreads) expand_pow2_kernel(ExpandArgs a, int32_t act_steps_per_grp, int32_t act_Kg) {
-    // (the status words are cleared by the host before this kernel: it may itself report a bad scale)
+    __shared__ __align__(16) uint8_t s_tab[kPow2Tables][16];
+    static_assert(kPow2Tables * 16 <= kExpandThreads, "one thread per table byte");
+    if (threadIdx.x < kPow2Tables * 16) {
+        const int s = (int)(threadIdx.x >> 4) + kPow2MinShift;
+        const float mul = __uint_as_float((uint32_t)((s > 0 ? s : 0) - 9 + 127) << 23);
+        s_tab[threadIdx.x >> 4][threadIdx.x & 15] = (uint8_t)pow2_bytes4(threadIdx.x & 15u, s < 0 ? -s : 0, mul);
+    }
+    __syncthreads();
+    pdl_trigger();                                         // the GEMM may set itself up meanwhile
+    if (blockIdx.x == 0 && threadIdx.x < 4) {
+        if (threadIdx.x == 0) {
+            const uint32_t keep = 11u | (*reinterpret_cast<volatile uint32_t*>(a.status + 2) << 8);
+            const uint32_t old = *reinterpret_cast<volatile uint32_t*>(a.status);
+            if (old != keep) atomicCAS(a.status, old, 0u);   // fails only if a report of this call came in between
+        } else if (threadIdx.x != 2) {
+            a.status[threadIdx.x] = 0u;
+        }
+    }
+    // one CTA takes a 128-row block and kPow2Chunks chunks of K-steps: thread t takes row t / 4 and, in every
+    // chunk, K-step t % 4, with all its loads issued before the first use
     const int piece = blockIdx.x;
-    const int blk = piece / a.n_chunks, kc = piece % a.n_chunks;
+    const int n_cp = (a.n_chunks + kPow2Chunks - 1) / kPow2Chunks;
+    const int blk = piece / n_cp, kc0 = (piece % n_cp) * kPow2Chunks;
     const int r = threadIdx.x >> 2;
-    const int ks = kc * kChunk + (threadIdx.x & 3);
-    if (ks >= a.n_steps) return;
     const bool is_a = blk < a.tiles_m;
     const int tile = is_a ? blk : blk - a.tiles_m;
     const int64_t row = (int64_t)tile * 128 + r;
     const int64_t rows = is_a ? a.M : a.O;
     const uint8_t* src = is_a ? a.xcodes : a.wcodes;
-    uint4 p = make_uint4(0, 0, 0, 0);
-    if (row < rows) p = __ldg(reinterpret_cast<const uint4*>(src + row * a.row_bytes + (int64_t)ks * 16));
-    uint4 c0, c1;
-    if (!is_a) {
-        expand8<false>(p.x, c0.x, c0.y);
-        expand8<false>(p.y, c0.z, c0.w);
-        expand8<false>(p.z, c1.x, c1.y);
-        expand8<false>(p.w, c1.z, c1.w);
-    } else {
-        int s = 0;
-        uint32_t row_scale = 0u;                           // bits of 2^e_m
-        if (row < rows) {
-            const float* sc = a.xscale + row * act_Kg;
-            uint32_t emax = 0u, bad = 0u;
-            int k = 0;
-            if ((act_Kg & 3) == 0 && (reinterpret_cast<uintptr_t>(sc) & 15) == 0) {   // four steps per load
-#pragma unroll 2
-                for (; k < act_Kg; k += 4) {
-                    const uint4 b4 = __ldg(reinterpret_cast<const uint4*>(sc + k));
-                    emax = max(max(emax, b4.x >> 23), max(max(b4.y >> 23, b4.z >> 23), b4.w >> 23));
-                    bad |= (b4.x | b4.y | b4.z | b4.w) & 0x807fffffu;
-                }
-            }
-            for (; k < act_Kg; ++k) {
-                const uint32_t bits = __float_as_uint(__ldg(sc + k));
-                emax = max(emax, bits >> 23);
-                bad |= bits & 0x807fffffu;                 // a mantissa or a sign: not a power of two
-            }
-            if (bad) atomicCAS(a.status, 0u, 11u | ((uint32_t)tile << 8));   // reported through the status word
-            const int e_m = (int)emax - 14;
-            s = (int)(__float_as_uint(__ldg(sc + ks / act_steps_per_grp)) >> 23) - e_m;
-            row_scale = e_m > 0 ? (uint32_t)e_m << 23 : 0u;
-        }
-        uint32_t w[8];
-        const uint32_t pw[4] = {p.x, p.y, p.z, p.w};
-        const int shr = s < 0 ? min(-s, 31) : 0;
-        const float mul = __uint_as_float((uint32_t)((s > 0 ? s : 0) - 9 + 127) << 23);
+    int ks[kPow2Chunks];
+    uint4 p[kPow2Chunks];
 #pragma unroll
-        for (int i = 0; i < 8; ++i)                        // four nibbles -> four bytes
-            w[i] = pow2_bytes4((pw[i >> 1] >> (16 * (i & 1))) & 0xffffu, shr, mul);
-        c0 = make_uint4(w[0], w[1], w[2], w[3]);
-        c1 = make_uint4(w[4], w[5], w[6], w[7]);
-        if (ks == 0) reinterpret_cast<uint32_t*>(a.s_blocks + (int64_t)tile * kScaleBlock)[r] = row_scale;
+    for (int j = 0; j < kPow2Chunks; ++j) {
+        ks[j] = (kc0 + j) * kChunk + (threadIdx.x & 3);
+        p[j] = make_uint4(0, 0, 0, 0);
+        if (row < rows && ks[j] < a.n_steps) p[j] = __ldg(reinterpret_cast<const uint4*>(src + row * a.row_bytes + (int64_t)ks[j] * 16));
     }
-    uint8_t* dst = (is_a ? a.a_blocks : a.b_blocks) + ((int64_t)tile * a.n_steps + ks) * kBlock;
-    const int off = (r >> 3) * 256 + (r & 7) * 16;
-    *reinterpret_cast<uint4*>(dst + off) = c0;
-    *reinterpret_cast<uint4*>(dst + off + 128) = c1;
+    int e_m = 0;
+    const float* sc = a.xscale + row * act_Kg;
+    if (is_a && row < rows) {
+        uint32_t emax = 0u, bad = 0u;
+        int k = 0;
+        if ((act_Kg & 3) == 0 && (reinterpret_cast<uintptr_t>(sc) & 15) == 0) {   // four steps per load
+#pragma unroll 2
+            for (; k < act_Kg; k += 4) {
+                const uint4 b4 = __ldg(reinterpret_cast<const uint4*>(sc + k));
+                emax = max(max(emax, b4.x >> 23), max(max(b4.y >> 23, b4.z >> 23), b4.w >> 23));
+                bad |= (b4.x | b4.y | b4.z | b4.w) & 0x807fffffu;
+            }
+        }
+        for (; k < act_Kg; ++k) {
+            const uint32_t bits = __float_as_uint(__ldg(sc + k));
+            emax = max(emax, bits >> 23);
+            bad |= bits & 0x807fffffu;                     // a mantissa or a sign: not a power of two
+        }
+        if (bad) atomicExch(a.status, 11u | (*reinterpret_cast<volatile uint32_t*>(a.status + 2) << 8));   // see above
+        e_m = (int)emax - 14;
+    }
+#pragma unroll
+    for (int j = 0; j < kPow2Chunks; ++j) {
+        if (ks[j] >= a.n_steps) break;
+        uint4 c0, c1;
+        if (!is_a) {
+            expand8<false>(p[j].x, c0.x, c0.y);
+            expand8<false>(p[j].y, c0.z, c0.w);
+            expand8<false>(p[j].z, c1.x, c1.y);
+            expand8<false>(p[j].w, c1.z, c1.w);
+        } else {
+            int s = 0;
+            if (row < rows) s = (int)(__float_as_uint(__ldg(sc + ks[j] / act_steps_per_grp)) >> 23) - e_m;
+            // s <= 14 by the choice of e_m (a step with its sign bit set is reported above; its bytes are not used)
+            const int ti = min(max(s, kPow2MinShift), 14) - kPow2MinShift;
+            const uint4 tab = *reinterpret_cast<const uint4*>(s_tab[ti]);
+            table_bytes8(p[j].x, tab, c0.x, c0.y);
+            table_bytes8(p[j].y, tab, c0.z, c0.w);
+            table_bytes8(p[j].z, tab, c1.x, c1.y);
+            table_bytes8(p[j].w, tab, c1.z, c1.w);
+            if (ks[j] == 0)                                // bits of 2^e_m, the row's one scale
+                reinterpret_cast<uint32_t*>(a.s_blocks + (int64_t)tile * kScaleBlock)[r] = row < rows && e_m > 0 ? (uint32_t)e_m << 23 : 0u;
+        }
+        uint8_t* dst = (is_a ? a.a_blocks : a.b_blocks) + ((int64_t)tile * a.n_steps + ks[j]) * kBlock;
+        const int off = (r >> 3) * 256 + (r & 7) * 16;
+        *reinterpret_cast<uint4*>(dst + off) = c0;
+        *reinterpret_cast<uint4*>(dst + off + 128) = c1;
+    }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -263,6 +318,7 @@ __global__ void __launch_bounds__(kThreads, 1) w4a4_gemm_kernel(const LinArgs a,
     tc_fence_after();
     pdl_wait();          // barrier set-up and the TMEM allocation overlap the tail of the kernel before this one
     pdl_trigger();
+    if (blockIdx.x == 0 && t == 0) atomicAdd(a.status + 2, 1u);   // the call's epoch (see expand_pow2_kernel)
     const uint32_t tmem_base = c->tmem_base;
 
     const int n_items = a.tiles_m * a.n_parts;
@@ -1196,12 +1252,14 @@ tdq_status linear_impl(const FusedSrc* fx, const uint8_t* xcodes, const float* x
 
     const unsigned pieces = (unsigned)((e.tiles_m + e.tiles_n) * p.n_chunks);
     if (pow2_steps) {
-        if (cudaMemsetAsync(workspace, 0, 16, stream) != cudaSuccess) return TDQ_ERR_CUDA;
-        expand_pow2_kernel<<<pieces, kExpandThreads, 0, stream>>>(e, act_group / 32, (int32_t)(I_pad / act_group));
+        const unsigned pieces2 = (unsigned)((e.tiles_m + e.tiles_n) * ((p.n_chunks + kPow2Chunks - 1) / kPow2Chunks));
+        expand_pow2_kernel<<<pieces2, kExpandThreads, 0, stream>>>(e, (int32_t)(act_group / 32), (int32_t)(I_pad / act_group));
     }
-    else if ((i8 ? launch_pdl(expand_kernel<true>, dim3(pieces), dim3(kExpandThreads), 0, stream, e)
-                 : launch_pdl(expand_kernel<false>, dim3(pieces), dim3(kExpandThreads), 0, stream, e)) != cudaSuccess)
-        return TDQ_ERR_CUDA;
+    else if (i8) expand_kernel<true><<<pieces, kExpandThreads, 0, stream>>>(e);
+    else expand_kernel<false><<<pieces, kExpandThreads, 0, stream>>>(e);
+    // (Ordinary launches: as programmatic dependents of the kernel before them the expansions were measured 1 to 4 us
+    // per call slower; their CTAs need next to no shared memory, so they can become resident beside a running GEMM
+    // and wait there.  The GEMM that follows is a programmatic dependent of the expansion: its set-up overlaps it.)
     if (cudaGetLastError() != cudaSuccess) return TDQ_ERR_CUDA;
     g_launch_count.fetch_add(1, std::memory_order_relaxed);
 

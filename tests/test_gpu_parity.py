@@ -478,6 +478,49 @@ def test_power_of_two_linear_truncation_bound_bf16_output_and_bad_scales(tdq):
     assert st != tdq.OK and (detail & 0xff) == 11
 
 
+@pytest.mark.gpu
+def test_power_of_two_bad_step_report_belongs_to_its_call(tdq):
+    # the report of a step that is not a power of two does not outlive its call: neither with one workspace
+    # used by call after call, nor when the calls are replays of one captured graph over changing scales
+    rng = np.random.RandomState(12)
+    M, C, O = 300, 256, 100
+    x = rng.normal(size=(M, C)).astype(np.float32)
+    w = (rng.normal(size=(O, C)) * 0.02).astype(np.float32)
+    good, bad = oracle.quantize_act(x, flags=7), oracle.quantize_act(x)
+    wq = oracle.quantize_weight(w)
+    codes, wc, ws = to_cuda(good["codes"]), to_cuda(wq["codes"]), to_cuda(wq["scale"])
+    s_good, s_bad = to_cuda(good["scale"]), to_cuda(bad["scale"])
+    wsp = torch.empty_like(tdq.linear_workspace(M, C, O, 32, "cuda")).fill_(0x5a)   # nothing relies on a cleared workspace
+    y = torch.empty((M, O), device="cuda")
+    scale = s_good.clone()
+
+    def status():
+        st, detail = tdq.workspace_status(wsp)
+        return 0 if st == tdq.OK else detail & 0xff
+
+    for want, src in [(0, s_good), (11, s_bad), (11, s_bad), (0, s_good), (0, s_good), (11, s_bad), (0, s_good)]:
+        scale.copy_(src)
+        tdq.w4a4_linear_pow2(codes, scale, wc, ws, y=y, workspace=wsp)
+        assert status() == want
+    y_good = y.clone()
+    # an exact-step call in between leaves nothing behind either
+    scale.copy_(s_bad)
+    tdq.w4a4_linear_pow2(codes, scale, wc, ws, y=y, workspace=wsp)
+    tdq.w4a4_linear(codes, scale, wc, ws, y=y, workspace=wsp)
+    assert status() == 0
+    tdq.w4a4_linear_pow2(codes, s_good, wc, ws, y=y, workspace=wsp)
+    assert status() == 0
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        tdq.w4a4_linear_pow2(codes, scale, wc, ws, y=y, workspace=wsp)
+    for want, src in [(11, s_bad), (0, s_good), (0, s_good), (11, s_bad), (11, s_bad), (0, s_good)]:
+        scale.copy_(src)
+        graph.replay()
+        assert status() == want
+    assert torch.equal(y.view(torch.int32), y_good.view(torch.int32))
+
+
 # ------------------------------------------------------------------------------------------
 # host-buffer entry point (chunked copies overlapped with the kernels)
 

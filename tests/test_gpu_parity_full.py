@@ -371,3 +371,37 @@ def test_group_sums_are_exact_on_extreme_codes(tdq, M, C, O, g):
         np.testing.assert_array_equal(acc.cpu().numpy().astype(np.int64), ref, err_msg=kind)
         # unit steps and unit channel scales: y is the integer sum over the groups, exact in binary32 below 2^24
         np.testing.assert_array_equal(y.cpu().numpy().astype(np.int64), ref.sum(axis=2), err_msg=kind)
+
+
+# ------------------------------------------------------------------------------------------
+# the power-of-two variant's operand bytes: every code value at every shift against the row's largest
+# step, the truncated ones included.  One-hot weight rows leave a single product per output, so every
+# expected value is exact in binary32 and the comparison is bit for bit.
+
+@pytest.mark.parametrize("C,g", [(128, 32), (256, 64), (256, 128), (768, 768)])
+def test_power_of_two_operand_is_exact_for_every_code_and_shift(tdq, C, g):
+    rng = np.random.RandomState(C + g)
+    M, O, Kg = 300, C, C // g
+    qx = ((np.arange(C)[None, :] + np.arange(M)[:, None] * 5) % 16 - 8).astype(np.int8)
+    drop = rng.randint(0, 22, size=(M, Kg))                # binades below the row's largest step
+    drop[np.arange(M), rng.randint(0, Kg, size=M)] = 0
+    drop[:23, 0] = 0
+    if Kg > 1:
+        drop[:23, 1] = np.arange(23)                       # every shift from 14 down to -8 occurs
+    top = rng.randint(-12, 6, size=(M, 1))
+    xs = np.exp2(top - drop).astype(np.float32)
+    qw = np.zeros((O, C), np.int8)
+    nz = np.array([7, -8, 1, -1, 3, -5, 6, -2, 4, -7], np.int8)
+    qw[np.arange(O), np.arange(C)] = nz[np.arange(O) % len(nz)]
+    ws = np.exp2(-(np.arange(O) % 5)).astype(np.float32)
+    wsp = tdq.linear_workspace(M, C, O, g, "cuda")
+    y = tdq.w4a4_linear_pow2(to_cuda(_pack_codes(qx)), to_cuda(xs), to_cuda(_pack_codes(qw)), to_cuda(ws), None,
+                             g=g, out_dtype=torch.float32, workspace=wsp)
+    st, detail = tdq.workspace_status(wsp)
+    assert st == tdq.OK, "status 0x%x" % detail
+    # s = 14 - drop; a code keeps |q| >> max(-s, 0) (towards zero) and its step
+    shr = np.maximum(drop - 14, 0).repeat(g, axis=1)
+    kept = np.sign(qx.astype(np.int64)) * (np.abs(qx.astype(np.int64)) >> shr)
+    v = kept.astype(np.float64) * np.exp2(shr) * xs.astype(np.float64).repeat(g, axis=1)
+    want = v * (np.diag(qw).astype(np.float64) * ws.astype(np.float64))[None, :]
+    np.testing.assert_array_equal(y.cpu().numpy().astype(np.float64), want)
