@@ -377,6 +377,26 @@ def small_configs_leg(tdq, dev, peaks):
     return out
 
 
+def pow2_leg(tdq, dev, workload_name):
+    """The power-of-two variant alone on a workload's shape: its quantizer once, then its linear layer from a graph."""
+    import torch
+    case = workload(workload_name)
+    M, C, O = case.M, case.C, case.w.shape[0]
+    x = torch.from_numpy(case.x.reshape(M, C).view(np.int16).copy()).view(torch.bfloat16).to(dev) if case.x_is_bf16 \
+        else torch.from_numpy(case.x.reshape(M, C)).to(dev)
+    wcodes, wscale = tdq.quantize_weight(torch.from_numpy(case.w).to(dev), 32)
+    p2 = tdq.act_params(flags=tdq.ENABLE_C1 | tdq.ENABLE_C2 | tdq.POW2_STEP)
+    codes, scale = tdq.quantize_act(x, p2)
+    ys = [torch.empty((M, O), dtype=torch.float32, device=dev) for _ in range(2)]
+    wsp = tdq.linear_workspace(M, C, O, 32, dev)
+    ms = time_graph(lambda i: tdq.w4a4_linear_pow2(codes, scale, wcodes, wscale, y=ys[i % 2], workspace=wsp), 8, replays=3)
+    st, detail = tdq.workspace_status(wsp)
+    if st != tdq.OK:
+        raise RuntimeError("tdq_w4a4_linear_pow2 reported 0x%x" % detail)
+    return dict(name="tdq_w4a4_linear_pow2", workload=workload_name, shape=[M, C, O], ms=ms,
+                tops=2.0 * M * C * O / (ms * 1e-3) / 1e12)
+
+
 def probe_leg(tdq, dev, peaks):
     """A compute-bound shape (16384 x 4096 -> 4096, bf16 output) with per-32 groups and with one group per token."""
     import torch
@@ -726,6 +746,7 @@ def main():
     ap.add_argument("--oracle-leg", type=int, default=0, help=argparse.SUPPRESS)
     ap.add_argument("--eager", action="store_true", help="launch every timed step from the host instead of replaying a CUDA graph")
     ap.add_argument("--probe-only", action="store_true", help="only the compute-bound probe shape of the linear layer (for profiler runs); prints that leg")
+    ap.add_argument("--pow2-only", action="store_true", help="only the power-of-two variant of the linear layer on --workload (for profiler runs); prints that leg")
     args = ap.parse_args()
     if args.oracle_leg:                    # child of cpu_oracle_single_thread
         print(json.dumps(cpu_oracle_leg(workload(args.workload), args.oracle_leg)))
@@ -734,6 +755,11 @@ def main():
         import torch
         from paper_2604_16855_b200 import tdq
         print(json.dumps(dict(compute_probe=probe_leg(tdq, torch.device("cuda", 0), load_peaks()))))
+        return
+    if args.pow2_only:
+        import torch
+        from paper_2604_16855_b200 import tdq
+        print(json.dumps(dict(w4a4_linear_pow2=pow2_leg(tdq, torch.device("cuda", 0), args.workload))))
         return
     if args.steps is None:
         args.steps = 10 if args.impl == "reference" else 1000
